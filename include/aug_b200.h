@@ -1,0 +1,202 @@
+/*
+ * aug_b200 -- on-GPU speech augmentation and feature extraction (sm_100a).
+ *
+ * What the paper's CPU "example servers" do to every utterance before it
+ * reaches a trainer (Sections 1 and 2.3: acoustic simulator with room
+ * configurations and impulse responses made on the fly, noise at a random SNR,
+ * VTLP with the bilinear warp of Eq. 1, mel filterbank features), done on one
+ * GPU:
+ *
+ *   1. aug_rir_image_method  room impulse responses of a shoebox room
+ *   2. aug_reverb_mix        reverberate speech and noise sources, mix at an SNR
+ *   3. feat_stft_power       framing, Hann window, power spectrum
+ *   4. feat_vtlp_logmel      warped mel filterbank, log (or power-law) compression
+ *   *  aug_pipeline          1-4 in one call, intermediates kept on the device
+ *
+ * Conventions shared by all calls
+ *   - Plain C ABI.  Every pointer is tagged `_dev` (device memory, caller-owned,
+ *     16-byte aligned) or `_host`.  The library never frees or keeps a caller
+ *     pointer beyond the kernels it enqueues.
+ *   - All device work of a context is enqueued on the CUDA stream given to
+ *     aug_create and the compute calls return without synchronising.  They
+ *     allocate nothing: the context owns a workspace sized at aug_create.
+ *   - Return value: AUG_OK (0) or a negative AugStatus.  Nothing throws, aborts
+ *     or traps.  Rows of the parameter table that a kernel has to reject are
+ *     recorded in a device status word, see aug_last_status.
+ *   - Audio is fp32 at AugConfig.fs; sample counts and frame counts are int32;
+ *     offsets into the noise bank are int64.
+ */
+#ifndef AUG_B200_H
+#define AUG_B200_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define AUG_S_MAX 4 /* speech + at most three noise sources per utterance */
+
+typedef enum {
+    AUG_OK = 0,
+    AUG_EINVAL = -1, /* null or misaligned pointer, bad scalar argument */
+    AUG_ECAP = -2,   /* batch, length, frames, taps or order beyond the context's capacity */
+    AUG_ECUDA = -3,  /* a CUDA runtime call or kernel launch failed */
+    AUG_EPARAM = -4, /* a parameter-table row failed validation */
+    AUG_ENOMEM = -5  /* workspace allocation failed in aug_create */
+} AugStatus;
+
+typedef enum { AUG_COMPRESS_LOG = 0, AUG_COMPRESS_POW_1_15 = 1 } AugCompression;
+
+/* Fixed at aug_create.  Plain data, no pointers. */
+typedef struct {
+    int32_t fs;              /* sampling rate, Hz */
+    int32_t win;             /* window length in samples (<= n_fft) */
+    int32_t hop;             /* frame shift in samples */
+    int32_t n_fft;           /* DFT size K: 512 or 1024 */
+    int32_t n_mel;           /* mel bands M, 1..128 */
+    float f_lo;              /* lowest filterbank edge, Hz */
+    float f_hi;              /* highest filterbank edge, Hz */
+    int32_t rir_taps;        /* L: taps of every impulse response, 1..24576 */
+    int32_t max_order;       /* largest reflection order a row may ask for, 0..32 */
+    int32_t max_sources;     /* 1..AUG_S_MAX */
+    int32_t frac_half_width; /* W_h of the windowed-sinc delay kernel, 1..47 */
+    float sound_speed;       /* m/s */
+    float log_floor;         /* filterbank energies are clamped to this before compression */
+    float pad_value;         /* written to feature rows at and beyond the frame count */
+    int32_t compression;     /* AugCompression */
+    int32_t max_batch;       /* capacity: utterances per call */
+    int32_t max_samples;     /* capacity: samples per utterance */
+    int32_t host_staging;    /* non-zero: also allocate device staging for aug_pipeline_host */
+    int64_t max_bank_samples; /* capacity of the staged noise bank (host_staging only) */
+} AugConfig;
+
+/*
+ * One row per utterance, 160 bytes.  Drawn on the HOST (the random room, SNR and
+ * warp factor of Sections 1 / 2.3) and copied to the device by the caller.
+ */
+typedef struct {
+    float room[3];                 /* shoebox side lengths, metres */
+    float beta[6];                 /* wall reflection coefficients in [0,1]: x=0, x=Lx, y=0, y=Ly, z=0, z=Lz */
+    float mic[3];                  /* microphone position */
+    int32_t n_src;                 /* 1 + number of noise sources, 1..max_sources */
+    int32_t order;                 /* keep images with |kx|+|ky|+|kz| <= order */
+    float snr_db;                  /* power of reverberant speech over power of summed reverberant noise */
+    float alpha;                   /* VTLP warp factor of Eq. 1, in (0,2); 1 = no warp */
+    float src_pos[AUG_S_MAX][3];   /* [0] = speech source, [1..] = noise sources */
+    int64_t noise_offset[AUG_S_MAX - 1]; /* start of this source's stretch of the noise bank */
+    int32_t noise_len[AUG_S_MAX - 1];    /* its length; it repeats end to end over the utterance */
+    float noise_weight[AUG_S_MAX - 1];   /* relative level of this source in the noise sum */
+} AugUttParams;
+
+typedef struct AugCtx AugCtx; /* opaque: configuration, tables, workspace */
+
+/* -------------------------------------------------------------- host-only helpers */
+
+/* Message for a status code; never NULL; static storage. */
+const char *aug_strerror(int code);
+
+/* Frames of an utterance of n_samples: 1 + (n_samples - win) / hop when
+ * n_samples >= win, else 0 (no padding, no centring).  Pure integer arithmetic;
+ * the kernels use the same expression. */
+int aug_frame_count(int n_samples, int win, int hop);
+
+/* Bytes of device workspace a context of this configuration allocates, or a
+ * negative AugStatus if the configuration is invalid. */
+int64_t aug_workspace_bytes(const AugConfig *cfg_host);
+
+/* Check B host rows against cfg: finite values, room sides > 0, microphone and
+ * sources inside the room and not coincident, beta in [0,1], alpha in (0,2),
+ * n_src in [1,max_sources], order in [0,max_order], noise stretches inside
+ * [0,bank_len) with positive length.  Returns AUG_OK or AUG_EPARAM with the index
+ * of the first bad row in *bad_row_host (may be NULL). */
+int aug_validate_params(const AugConfig *cfg_host, const AugUttParams *table_host, int B,
+                        int64_t bank_len, int *bad_row_host);
+
+/* -------------------------------------------------------------- context */
+
+/* Create a context for cfg on the current CUDA device; cuda_stream is a
+ * cudaStream_t (NULL = default stream).  All allocation happens here.
+ * On failure *out is NULL. */
+int aug_create(AugCtx **out, const AugConfig *cfg_host, void *cuda_stream);
+
+/* Waits for the context's stream, frees the workspace.  NULL is accepted. */
+int aug_destroy(AugCtx *ctx);
+
+/* Synchronises the context's stream and reads the device status word.
+ * *utt_host = first utterance a kernel rejected (-1 if none), *reason_host =
+ * 1 n_src out of range, 2 order out of range, 3 bad noise stretch, 4 a bounded
+ * wait inside a kernel ran out.  A rejected utterance gets zero impulse
+ * responses / silent output; nothing faults.  The word is cleared by the read. */
+int aug_last_status(AugCtx *ctx, int *utt_host, int *reason_host);
+
+/* -------------------------------------------------------------- step 1
+ * Room impulse responses by the image-source method (simulator block, Sections
+ * 1 and 2.3; computed on the fly per utterance as Section 1 requires).
+ *   rir_dev [B][max_sources][rir_taps] fp32, overwritten; sources >= n_src get zeros.
+ * For each source the sum runs over the image lattice |kx|+|ky|+|kz| <= order;
+ * an image at distance d adds (prod beta^hits / d) times a Hann-windowed sinc
+ * (half width frac_half_width) centred at d*fs/sound_speed samples. */
+int aug_rir_image_method(AugCtx *ctx, const AugUttParams *table_dev, int B, float *rir_dev);
+
+/* -------------------------------------------------------------- step 2
+ * Reverberation and noise mixing (simulator block, Sections 1 and 2.3).
+ *   speech_dev  [B][speech_stride] fp32; speech_stride a multiple of 4
+ *   lengths_dev [B] int32, 0 <= lengths[b] <= min(speech_stride, max_samples)
+ *   noise_bank_dev [bank_len] fp32 (may be NULL when no row has noise)
+ *   rir_dev     as written by step 1
+ *   wave_out_dev [B][speech_stride] fp32: samples [0,lengths[b]) written,
+ *               the rest of each row left untouched
+ * y_s = speech * rir[0] and v = sum_k weight_k (noise_k * rir[k]) are causal
+ * convolutions cut to the utterance length, done as FFT overlap convolution;
+ * out = y_s + g v with g = sqrt(sum y_s^2 / (sum v^2 10^(snr_db/10))), g = 0 when
+ * there is no noise or either sum is zero. */
+int aug_reverb_mix(AugCtx *ctx, const float *speech_dev, int64_t speech_stride,
+                   const int *lengths_dev, const float *noise_bank_dev, int64_t bank_len,
+                   const float *rir_dev, const AugUttParams *table_dev, int B,
+                   float *wave_out_dev);
+
+/* -------------------------------------------------------------- step 3
+ * Framing, periodic Hann window and power spectrum (feature block, Section 2.3).
+ *   wave_dev  [B][stride] fp32;  power_dev [B][T_max][n_fft/2+1] fp32
+ *   frame_counts_dev [B] int32 = min(aug_frame_count(lengths[b]), T_max)
+ * P[t][k] = |sum_{n<win} hann[n] wave[t hop + n] exp(-2 pi i k n / n_fft)|^2, no
+ * scaling.  Rows t >= frame count are set to zero. */
+int feat_stft_power(AugCtx *ctx, const float *wave_dev, int64_t stride, const int *lengths_dev,
+                    int B, float *power_dev, int T_max, int *frame_counts_dev);
+
+/* -------------------------------------------------------------- step 4
+ * Mel filterbank with the VTLP warp of Eq. 1 and compression (Section 2.3).
+ *   feats_dev [B][T_max][n_mel] fp32
+ * Triangles are linear in mel (2595 log10(1+f/700)), peak 1, edges equally spaced
+ * from f_lo to f_hi, evaluated at the warped frequency of each DFT bin
+ * (omega' of Eq. 1 with the row's alpha).  feat = ln(max(E, log_floor)), or
+ * max(E, log_floor)^(1/15) for AUG_COMPRESS_POW_1_15.  Rows t >= frame_counts[b]
+ * receive pad_value. */
+int feat_vtlp_logmel(AugCtx *ctx, const float *power_dev, const int *frame_counts_dev,
+                     const AugUttParams *table_dev, int B, int T_max, float *feats_dev);
+
+/* -------------------------------------------------------------- steps 1-4
+ * The whole path for a batch.  Arguments as above; additionally
+ *   lengths_host  the same lengths in host memory (may be NULL): used only to size
+ *                 launches tightly and to check capacities without a device sync
+ *   wave_out_dev_or_null  if not NULL, also receives the mixed waveform as in step 2
+ * Writes feats_dev [B][T_max][n_mel] (padded with pad_value) and frame_counts_dev. */
+int aug_pipeline(AugCtx *ctx, const float *speech_dev, int64_t speech_stride,
+                 const int *lengths_dev, const int *lengths_host, const float *noise_bank_dev,
+                 int64_t bank_len, const AugUttParams *table_dev, int B, float *feats_dev,
+                 int T_max, int *frame_counts_dev, float *wave_out_dev_or_null);
+
+/* Same call for callers that hold HOST buffers: copies speech, lengths, noise
+ * bank and table to device staging owned by the context, runs the path, copies
+ * feats and frame counts back and synchronises.  Host buffers should be pinned
+ * for full copy bandwidth. */
+int aug_pipeline_host(AugCtx *ctx, const float *speech_host, int64_t speech_stride,
+                      const int *lengths_host, const float *noise_bank_host, int64_t bank_len,
+                      const AugUttParams *table_host, int B, float *feats_host, int T_max,
+                      int *frame_counts_host);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AUG_B200_H */

@@ -1,0 +1,350 @@
+// C ABI of libaugb200: argument checks, context and workspace, call sequencing.
+#include <math.h>
+#include <new>
+#include <stdlib.h>
+#include <string.h>
+#include <vector>
+
+#include "common.cuh"
+#include "fft.cuh"
+
+namespace {
+
+inline int64_t align_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_config(const AugConfig *c) {
+    if (!c) return AUG_EINVAL;
+    if (c->fs <= 0 || c->hop <= 0 || c->win <= 0) return AUG_EINVAL;
+    if (c->n_fft != 512 && c->n_fft != 1024) return AUG_EINVAL;
+    if (c->win > c->n_fft) return AUG_EINVAL;
+    if (c->n_mel < 1 || c->n_mel > aug::MAX_MEL) return AUG_EINVAL;
+    if (!(c->f_lo >= 0.f) || !(c->f_hi > c->f_lo) || c->f_hi > 0.5f * c->fs + 1e-3f) return AUG_EINVAL;
+    if (c->rir_taps < 1 || c->rir_taps > aug::MAX_TAPS) return AUG_EINVAL;
+    if (c->max_order < 0 || c->max_order > aug::MAX_ORDER) return AUG_EINVAL;
+    if (c->max_sources < 1 || c->max_sources > AUG_S_MAX) return AUG_EINVAL;
+    if (c->frac_half_width < 1 || c->frac_half_width > aug::MAX_HALF_W) return AUG_EINVAL;
+    if (!(c->sound_speed > 0.f) || !(c->log_floor > 0.f) || !isfinite(c->pad_value)) return AUG_EINVAL;
+    if (c->compression != AUG_COMPRESS_LOG && c->compression != AUG_COMPRESS_POW_1_15) return AUG_EINVAL;
+    if (c->max_batch < 1 || c->max_batch > 65535 || c->max_samples < 1) return AUG_EINVAL;
+    if (c->host_staging && c->max_bank_samples < 0) return AUG_EINVAL;
+    return AUG_OK;
+}
+
+struct Layout {
+    int n_part, n_bins, t_cap;
+    int64_t ws_stride;
+    int64_t off_tw, off_rir, off_hspec, off_ys, off_vv, off_energy, off_melw, off_melstart,
+        off_status, off_counts, off_st_speech, off_st_bank, off_st_table, off_st_lengths,
+        off_st_feats, off_st_counts, total;
+};
+
+Layout make_layout(const AugConfig &c) {
+    Layout l;
+    l.n_part = (c.rir_taps + aug::CONV_BLK - 1) / aug::CONV_BLK;
+    l.n_bins = c.n_fft / 2 + 1;
+    l.t_cap = aug_frame_count(c.max_samples, c.win, c.hop);
+    l.ws_stride = align_up(c.max_samples, 4);
+    const int64_t B = c.max_batch, S = c.max_sources;
+    int64_t o = 0;
+    auto take = [&](int64_t bytes) { int64_t r = o; o = align_up(o + bytes, 256); return r; };
+    l.off_tw = take(sizeof(float2) * augfft::TW_N);
+    l.off_rir = take(sizeof(float) * B * S * c.rir_taps);
+    l.off_hspec = take(sizeof(float2) * B * S * l.n_part * aug::CONV_N2);
+    l.off_ys = take(sizeof(float) * B * l.ws_stride);
+    l.off_vv = take(sizeof(float) * B * l.ws_stride);
+    l.off_energy = take(sizeof(double) * 2 * B);
+    l.off_melw = take(sizeof(aug::MelBin) * B * l.n_bins);
+    l.off_melstart = take(sizeof(int) * B * (c.n_mel + 2));
+    l.off_status = take(sizeof(int) * 2);
+    l.off_counts = take(sizeof(int) * B);
+    if (c.host_staging) {
+        l.off_st_speech = take(sizeof(float) * B * l.ws_stride);
+        l.off_st_bank = take(sizeof(float) * (c.max_bank_samples > 0 ? c.max_bank_samples : 1));
+        l.off_st_table = take(sizeof(AugUttParams) * B);
+        l.off_st_lengths = take(sizeof(int) * B);
+        l.off_st_feats = take(sizeof(float) * B * (int64_t)(l.t_cap > 0 ? l.t_cap : 1) * c.n_mel);
+        l.off_st_counts = take(sizeof(int) * B);
+    } else {
+        l.off_st_speech = l.off_st_bank = l.off_st_table = l.off_st_lengths = l.off_st_feats =
+            l.off_st_counts = -1;
+    }
+    l.total = o;
+    return l;
+}
+
+// Common checks of the batch arguments; max_len_out = largest length if known from the host.
+int check_batch(const AugCtx *ctx, int B) {
+    if (!ctx) return AUG_EINVAL;
+    if (B < 0) return AUG_EINVAL;
+    if (B > ctx->cfg.max_batch) return AUG_ECAP;
+    return AUG_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *aug_strerror(int code) {
+    switch (code) {
+        case AUG_OK: return "success";
+        case AUG_EINVAL: return "invalid argument (null or misaligned pointer, bad scalar)";
+        case AUG_ECAP: return "request exceeds the capacity the context was created with";
+        case AUG_ECUDA: return "CUDA runtime call or kernel launch failed";
+        case AUG_EPARAM: return "parameter table row failed validation";
+        case AUG_ENOMEM: return "device workspace allocation failed";
+        default: return "unknown status code";
+    }
+}
+
+int aug_frame_count(int n_samples, int win, int hop) {
+    if (win <= 0 || hop <= 0 || n_samples < win) return 0;
+    return 1 + (n_samples - win) / hop;
+}
+
+int64_t aug_workspace_bytes(const AugConfig *cfg) {
+    int rc = check_config(cfg);
+    if (rc != AUG_OK) return rc;
+    return make_layout(*cfg).total;
+}
+
+int aug_validate_params(const AugConfig *cfg, const AugUttParams *tab, int B, int64_t bank_len,
+                        int *bad_row) {
+    if (bad_row) *bad_row = -1;
+    if (!cfg || (!tab && B > 0) || B < 0) return AUG_EINVAL;
+    for (int b = 0; b < B; ++b) {
+        const AugUttParams &r = tab[b];
+        bool ok = r.n_src >= 1 && r.n_src <= cfg->max_sources && r.order >= 0 &&
+                  r.order <= cfg->max_order && isfinite(r.snr_db) && r.alpha > 0.f && r.alpha < 2.f;
+        for (int a = 0; a < 3 && ok; ++a) {
+            ok = isfinite(r.room[a]) && r.room[a] > 0.f && r.mic[a] >= 0.f && r.mic[a] <= r.room[a];
+        }
+        for (int w = 0; w < 6 && ok; ++w) ok = r.beta[w] >= 0.f && r.beta[w] <= 1.f;
+        for (int s = 0; s < r.n_src && ok; ++s) {
+            double d2 = 0.0;
+            for (int a = 0; a < 3 && ok; ++a) {
+                const float p = r.src_pos[s][a];
+                ok = p >= 0.f && p <= r.room[a];
+                d2 += ((double)p - r.mic[a]) * ((double)p - r.mic[a]);
+            }
+            if (ok) ok = d2 > 1e-12;   // a source on top of the microphone has no finite 1/d
+        }
+        for (int k = 0; k + 1 < r.n_src && ok; ++k) {
+            ok = r.noise_len[k] > 0 && r.noise_offset[k] >= 0 &&
+                 r.noise_offset[k] + r.noise_len[k] <= bank_len && isfinite(r.noise_weight[k]);
+        }
+        if (!ok) {
+            if (bad_row) *bad_row = b;
+            return AUG_EPARAM;
+        }
+    }
+    return AUG_OK;
+}
+
+int aug_create(AugCtx **out, const AugConfig *cfg, void *cuda_stream) {
+    if (!out) return AUG_EINVAL;
+    *out = nullptr;
+    int rc = check_config(cfg);
+    if (rc != AUG_OK) return rc;
+    AugCtx *ctx = new (std::nothrow) AugCtx();
+    if (!ctx) return AUG_ENOMEM;
+    memset(ctx, 0, sizeof(*ctx));
+    ctx->cfg = *cfg;
+    ctx->stream = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaGetDevice(&ctx->device) != cudaSuccess) {
+        delete ctx;
+        return AUG_ECUDA;
+    }
+    const Layout l = make_layout(*cfg);
+    ctx->n_part = l.n_part;
+    ctx->n_bins = l.n_bins;
+    ctx->t_cap = l.t_cap;
+    ctx->ws_stride = l.ws_stride;
+    ctx->ws_bytes = l.total;
+    if (cudaMalloc(&ctx->ws_base, (size_t)l.total) != cudaSuccess) {
+        cudaGetLastError();
+        delete ctx;
+        return AUG_ENOMEM;
+    }
+    char *base = static_cast<char *>(ctx->ws_base);
+    ctx->tw = reinterpret_cast<float2 *>(base + l.off_tw);
+    ctx->rir = reinterpret_cast<float *>(base + l.off_rir);
+    ctx->hspec = reinterpret_cast<float2 *>(base + l.off_hspec);
+    ctx->ys = reinterpret_cast<float *>(base + l.off_ys);
+    ctx->vv = reinterpret_cast<float *>(base + l.off_vv);
+    ctx->energy = reinterpret_cast<double *>(base + l.off_energy);
+    ctx->melw = reinterpret_cast<aug::MelBin *>(base + l.off_melw);
+    ctx->melstart = reinterpret_cast<int *>(base + l.off_melstart);
+    ctx->status = reinterpret_cast<int *>(base + l.off_status);
+    ctx->counts_tmp = reinterpret_cast<int *>(base + l.off_counts);
+    if (cfg->host_staging) {
+        ctx->st_speech = reinterpret_cast<float *>(base + l.off_st_speech);
+        ctx->st_bank = reinterpret_cast<float *>(base + l.off_st_bank);
+        ctx->st_table = reinterpret_cast<AugUttParams *>(base + l.off_st_table);
+        ctx->st_lengths = reinterpret_cast<int *>(base + l.off_st_lengths);
+        ctx->st_feats = reinterpret_cast<float *>(base + l.off_st_feats);
+        ctx->st_counts = reinterpret_cast<int *>(base + l.off_st_counts);
+    }
+    // twiddles exp(-2 pi i m / TW_N), evaluated in double
+    std::vector<float2> tw(augfft::TW_N);
+    for (int m = 0; m < augfft::TW_N; ++m) {
+        const double a = -2.0 * 3.14159265358979323846 * m / augfft::TW_N;
+        tw[m] = make_float2((float)cos(a), (float)sin(a));
+    }
+    const int st0[2] = {-1, 0};
+    bool ok = cudaMemcpyAsync(ctx->tw, tw.data(), sizeof(float2) * augfft::TW_N,
+                              cudaMemcpyHostToDevice, ctx->stream) == cudaSuccess &&
+              cudaMemcpyAsync(ctx->status, st0, sizeof(st0), cudaMemcpyHostToDevice,
+                              ctx->stream) == cudaSuccess &&
+              cudaStreamSynchronize(ctx->stream) == cudaSuccess;
+    if (!ok) {
+        cudaFree(ctx->ws_base);
+        delete ctx;
+        return AUG_ECUDA;
+    }
+    *out = ctx;
+    return AUG_OK;
+}
+
+int aug_destroy(AugCtx *ctx) {
+    if (!ctx) return AUG_OK;
+    int rc = AUG_OK;
+    if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) rc = AUG_ECUDA;
+    if (cudaFree(ctx->ws_base) != cudaSuccess) rc = AUG_ECUDA;
+    delete ctx;
+    return rc;
+}
+
+int aug_last_status(AugCtx *ctx, int *utt, int *reason) {
+    if (!ctx) return AUG_EINVAL;
+    int st[2] = {-1, 0};
+    AUG_CUDA_OK(cudaMemcpyAsync(st, ctx->status, sizeof(st), cudaMemcpyDeviceToHost, ctx->stream));
+    AUG_CUDA_OK(cudaStreamSynchronize(ctx->stream));
+    const int clear[2] = {-1, 0};
+    AUG_CUDA_OK(cudaMemcpyAsync(ctx->status, clear, sizeof(clear), cudaMemcpyHostToDevice, ctx->stream));
+    AUG_CUDA_OK(cudaStreamSynchronize(ctx->stream));
+    if (utt) *utt = st[0];
+    if (reason) *reason = st[0] >= 0 ? st[1] : 0;
+    return AUG_OK;
+}
+
+int aug_rir_image_method(AugCtx *ctx, const AugUttParams *table_dev, int B, float *rir_dev) {
+    int rc = check_batch(ctx, B);
+    if (rc != AUG_OK) return rc;
+    if (B == 0) return AUG_OK;
+    if (!table_dev || !rir_dev || !aligned16(rir_dev)) return AUG_EINVAL;
+    return launch_rir(ctx, table_dev, B, rir_dev);
+}
+
+int aug_reverb_mix(AugCtx *ctx, const float *speech_dev, int64_t speech_stride,
+                   const int *lengths_dev, const float *noise_bank_dev, int64_t bank_len,
+                   const float *rir_dev, const AugUttParams *table_dev, int B, float *wave_out_dev) {
+    int rc = check_batch(ctx, B);
+    if (rc != AUG_OK) return rc;
+    if (B == 0) return AUG_OK;
+    if (!speech_dev || !lengths_dev || !rir_dev || !table_dev || !wave_out_dev) return AUG_EINVAL;
+    if (!aligned16(speech_dev) || !aligned16(wave_out_dev) || !aligned16(rir_dev)) return AUG_EINVAL;
+    if (noise_bank_dev && !aligned16(noise_bank_dev)) return AUG_EINVAL;
+    if (speech_stride <= 0 || (speech_stride & 3) || bank_len < 0) return AUG_EINVAL;
+    const int max_len = (int)(speech_stride < ctx->cfg.max_samples ? speech_stride : ctx->cfg.max_samples);
+    if (speech_stride > ctx->ws_stride) return AUG_ECAP;
+    if ((rc = launch_rir_spectra(ctx, rir_dev, table_dev, B)) != AUG_OK) return rc;
+    if ((rc = launch_convolve(ctx, speech_dev, speech_stride, lengths_dev, noise_bank_dev, bank_len,
+                              table_dev, B, max_len)) != AUG_OK) return rc;
+    return launch_mix(ctx, lengths_dev, table_dev, B, max_len, wave_out_dev, speech_stride);
+}
+
+int feat_stft_power(AugCtx *ctx, const float *wave_dev, int64_t stride, const int *lengths_dev,
+                    int B, float *power_dev, int T_max, int *frame_counts_dev) {
+    int rc = check_batch(ctx, B);
+    if (rc != AUG_OK) return rc;
+    if (B == 0) return AUG_OK;
+    if (!wave_dev || !lengths_dev || !power_dev || !frame_counts_dev) return AUG_EINVAL;
+    if (!aligned16(wave_dev) || stride <= 0 || T_max < 0) return AUG_EINVAL;
+    if (T_max == 0) return AUG_EINVAL;
+    return launch_stft_power(ctx, wave_dev, stride, lengths_dev, B, power_dev, T_max, frame_counts_dev);
+}
+
+int feat_vtlp_logmel(AugCtx *ctx, const float *power_dev, const int *frame_counts_dev,
+                     const AugUttParams *table_dev, int B, int T_max, float *feats_dev) {
+    int rc = check_batch(ctx, B);
+    if (rc != AUG_OK) return rc;
+    if (B == 0) return AUG_OK;
+    if (!power_dev || !frame_counts_dev || !table_dev || !feats_dev || T_max <= 0) return AUG_EINVAL;
+    if ((rc = launch_mel_tables(ctx, table_dev, B)) != AUG_OK) return rc;
+    return launch_logmel(ctx, power_dev, frame_counts_dev, B, T_max, feats_dev);
+}
+
+int aug_pipeline(AugCtx *ctx, const float *speech_dev, int64_t speech_stride,
+                 const int *lengths_dev, const int *lengths_host, const float *noise_bank_dev,
+                 int64_t bank_len, const AugUttParams *table_dev, int B, float *feats_dev,
+                 int T_max, int *frame_counts_dev, float *wave_out) {
+    int rc = check_batch(ctx, B);
+    if (rc != AUG_OK) return rc;
+    if (B == 0) return AUG_OK;
+    if (!speech_dev || !lengths_dev || !table_dev || !feats_dev || !frame_counts_dev) return AUG_EINVAL;
+    if (!aligned16(speech_dev) || !aligned16(feats_dev)) return AUG_EINVAL;
+    if (noise_bank_dev && !aligned16(noise_bank_dev)) return AUG_EINVAL;
+    if (wave_out && !aligned16(wave_out)) return AUG_EINVAL;
+    if (speech_stride <= 0 || (speech_stride & 3) || bank_len < 0 || T_max <= 0) return AUG_EINVAL;
+    if (speech_stride > ctx->ws_stride) return AUG_ECAP;
+    int max_len = (int)(speech_stride < ctx->cfg.max_samples ? speech_stride : ctx->cfg.max_samples);
+    if (lengths_host) {
+        int mx = 0;
+        for (int b = 0; b < B; ++b) {
+            if (lengths_host[b] < 0) return AUG_EINVAL;
+            if (lengths_host[b] > max_len) return AUG_ECAP;
+            if (lengths_host[b] > mx) mx = lengths_host[b];
+        }
+        if (aug_frame_count(mx, ctx->cfg.win, ctx->cfg.hop) > T_max) return AUG_ECAP;
+        max_len = mx;
+    }
+    if ((rc = launch_rir(ctx, table_dev, B, ctx->rir)) != AUG_OK) return rc;
+    if ((rc = launch_rir_spectra(ctx, ctx->rir, table_dev, B)) != AUG_OK) return rc;
+    if ((rc = launch_mel_tables(ctx, table_dev, B)) != AUG_OK) return rc;
+    if ((rc = launch_convolve(ctx, speech_dev, speech_stride, lengths_dev, noise_bank_dev, bank_len,
+                              table_dev, B, max_len)) != AUG_OK) return rc;
+    if (wave_out &&
+        (rc = launch_mix(ctx, lengths_dev, table_dev, B, max_len, wave_out, speech_stride)) != AUG_OK)
+        return rc;
+    return launch_fused_features(ctx, lengths_dev, table_dev, B, feats_dev, T_max, frame_counts_dev,
+                                 nullptr, 0);
+}
+
+int aug_pipeline_host(AugCtx *ctx, const float *speech_host, int64_t speech_stride,
+                      const int *lengths_host, const float *noise_bank_host, int64_t bank_len,
+                      const AugUttParams *table_host, int B, float *feats_host, int T_max,
+                      int *frame_counts_host) {
+    int rc = check_batch(ctx, B);
+    if (rc != AUG_OK) return rc;
+    if (!ctx->st_speech) return AUG_EINVAL;   // context created without host_staging
+    if (B == 0) return AUG_OK;
+    if (!speech_host || !lengths_host || !table_host || !feats_host || !frame_counts_host) return AUG_EINVAL;
+    if (speech_stride <= 0 || (speech_stride & 3) || bank_len < 0 || T_max <= 0) return AUG_EINVAL;
+    if (speech_stride > ctx->ws_stride || bank_len > ctx->cfg.max_bank_samples || T_max > ctx->t_cap)
+        return AUG_ECAP;
+    if (bank_len > 0 && !noise_bank_host) return AUG_EINVAL;
+    cudaStream_t st = ctx->stream;
+    AUG_CUDA_OK(cudaMemcpyAsync(ctx->st_speech, speech_host, sizeof(float) * (size_t)B * speech_stride,
+                                cudaMemcpyHostToDevice, st));
+    if (bank_len > 0)
+        AUG_CUDA_OK(cudaMemcpyAsync(ctx->st_bank, noise_bank_host, sizeof(float) * (size_t)bank_len,
+                                    cudaMemcpyHostToDevice, st));
+    AUG_CUDA_OK(cudaMemcpyAsync(ctx->st_table, table_host, sizeof(AugUttParams) * (size_t)B,
+                                cudaMemcpyHostToDevice, st));
+    AUG_CUDA_OK(cudaMemcpyAsync(ctx->st_lengths, lengths_host, sizeof(int) * (size_t)B,
+                                cudaMemcpyHostToDevice, st));
+    rc = aug_pipeline(ctx, ctx->st_speech, speech_stride, ctx->st_lengths, lengths_host,
+                      bank_len > 0 ? ctx->st_bank : nullptr, bank_len, ctx->st_table, B,
+                      ctx->st_feats, T_max, ctx->st_counts, nullptr);
+    if (rc != AUG_OK) return rc;
+    AUG_CUDA_OK(cudaMemcpyAsync(feats_host, ctx->st_feats,
+                                sizeof(float) * (size_t)B * T_max * ctx->cfg.n_mel,
+                                cudaMemcpyDeviceToHost, st));
+    AUG_CUDA_OK(cudaMemcpyAsync(frame_counts_host, ctx->st_counts, sizeof(int) * (size_t)B,
+                                cudaMemcpyDeviceToHost, st));
+    AUG_CUDA_OK(cudaStreamSynchronize(st));
+    return AUG_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,80 @@
+// Internal declarations shared by the translation units of libaugb200.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/aug_b200.h"
+
+namespace aug {
+
+constexpr int CONV_BLK = 4096;          // output samples per convolution block
+constexpr int CONV_F = 2 * CONV_BLK;    // real FFT size of one block
+constexpr int CONV_N2 = CONV_F / 2;     // complex FFT size
+constexpr int MAX_TAPS = 24576;
+constexpr int MAX_ORDER = 32;
+constexpr int MAX_HALF_W = 47;
+constexpr int MAX_MEL = 128;
+
+enum Reason { R_NONE = 0, R_NSRC = 1, R_ORDER = 2, R_NOISE = 3, R_WAIT = 4 };
+
+// Per-bin entry of the warped filterbank: the bin lies in edge interval `seg`
+// (between edges e_seg and e_seg+1), at fraction `up` from its lower edge.
+struct MelBin {
+    float up;    // weight in filter seg   (rising side)
+    float down;  // weight in filter seg-1 (falling side) = 1 - up
+};
+
+}  // namespace aug
+
+struct AugCtx {
+    AugConfig cfg;
+    cudaStream_t stream;
+    int device;
+    int n_part;            // RIR partitions of CONV_BLK taps
+    int n_bins;            // n_fft/2 + 1
+    int t_cap;             // frames of an utterance of max_samples
+    int64_t ws_stride;     // row stride (floats) of the y_s / v workspaces
+    // device workspace (one allocation, carved up)
+    void *ws_base;
+    int64_t ws_bytes;
+    float2 *tw;            // [TW_N] twiddles
+    float *rir;            // [max_batch][max_sources][rir_taps]
+    float2 *hspec;         // [max_batch][max_sources][n_part][CONV_N2]
+    float *ys;             // [max_batch][ws_stride]
+    float *vv;             // [max_batch][ws_stride]
+    double *energy;        // [max_batch][2]
+    aug::MelBin *melw;     // [max_batch][n_bins]
+    int *melstart;         // [max_batch][n_mel + 2]
+    int *status;           // [2]: utterance, reason
+    int *counts_tmp;       // [max_batch]
+    // staging for the host-buffer entry point (NULL unless cfg.host_staging)
+    float *st_speech;      // [max_batch][ws_stride]
+    float *st_bank;        // [max_bank_samples]
+    AugUttParams *st_table;
+    int *st_lengths;
+    float *st_feats;       // [max_batch][t_cap][n_mel]
+    int *st_counts;
+};
+
+#define AUG_CUDA_OK(expr)                         \
+    do {                                          \
+        cudaError_t e__ = (expr);                 \
+        if (e__ != cudaSuccess) return AUG_ECUDA; \
+    } while (0)
+
+// Launchers (defined next to their kernels).  All enqueue on ctx->stream.
+int launch_rir(AugCtx *ctx, const AugUttParams *table, int B, float *rir);
+int launch_rir_spectra(AugCtx *ctx, const float *rir, const AugUttParams *table, int B);
+int launch_convolve(AugCtx *ctx, const float *speech, int64_t stride, const int *lengths,
+                    const float *bank, int64_t bank_len, const AugUttParams *table, int B,
+                    int max_len);
+int launch_mix(AugCtx *ctx, const int *lengths, const AugUttParams *table, int B, int max_len,
+               float *wave_out, int64_t out_stride);
+int launch_mel_tables(AugCtx *ctx, const AugUttParams *table, int B);
+int launch_stft_power(AugCtx *ctx, const float *wave, int64_t stride, const int *lengths, int B,
+                      float *power, int T_max, int *counts);
+int launch_logmel(AugCtx *ctx, const float *power, const int *counts, int B, int T_max,
+                  float *feats);
+int launch_fused_features(AugCtx *ctx, const int *lengths, const AugUttParams *table, int B,
+                          float *feats, int T_max, int *counts, float *wave_out,
+                          int64_t out_stride);

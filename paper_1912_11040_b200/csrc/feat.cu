@@ -1,0 +1,336 @@
+// Steps 3 and 4: framing, Hann window, power spectrum, VTLP-warped mel
+// filterbank and compression -- separately (stft_power / logmel kernels) and
+// fused with the SNR mix (fused kernel: y_s + g v -> features, the power
+// spectrum never leaves shared memory).
+//
+// A CTA owns a tile of FT consecutive frames of one utterance.  It stages the
+// contiguous stretch of samples those frames cover in shared memory once, then
+// groups of 64 threads transform two frames at a time as the real and imaginary
+// part of one complex K-point FFT and separate the two spectra afterwards.
+// The filterbank is applied as a gather: band m sums the bins of edge interval m
+// with their rising weights and those of interval m+1 with their falling
+// weights; the intervals are contiguous bin ranges because the warp of Eq. 1 is
+// monotone.
+#include "common.cuh"
+#include "fft.cuh"
+
+namespace {
+
+using namespace augfft;
+constexpr int FEAT_THREADS = 256;
+constexpr int GROUP = 64;                         // threads per FFT
+constexpr int NGROUP = FEAT_THREADS / GROUP;
+
+__host__ __device__ __forceinline__ int frame_count(int n, int win, int hop) {
+    return n >= win ? 1 + (n - win) / hop : 0;
+}
+
+// ---------------------------------------------------------------- filterbank tables
+// One CTA per utterance: per DFT bin the edge interval and weights at the warped
+// frequency (fp64: a bin that barely enters a band must not lose its weight to
+// rounding), then the first bin of every interval.
+__global__ void __launch_bounds__(256)
+mel_tables_kernel(const AugUttParams *__restrict__ table, int K, int M, double fs, double f_lo,
+                  double f_hi, aug::MelBin *__restrict__ melw, int *__restrict__ melstart) {
+    __shared__ int seg_s[513];
+    const int utt = blockIdx.x, nb = K / 2 + 1;
+    const double a = 1.0 - (double)table[utt].alpha;
+    const double PI = 3.14159265358979323846;
+    const double e0 = 2595.0 * log10(1.0 + f_lo / 700.0);
+    const double e1 = 2595.0 * log10(1.0 + f_hi / 700.0);
+    const double delta = (e1 - e0) / (M + 1);
+    for (int k = threadIdx.x; k < nb; k += blockDim.x) {
+        const double om = 2.0 * PI * k / K;
+        const double omw = om + 2.0 * atan(a * sin(om) / (1.0 - a * cos(om)));   // Eq. 1
+        const double fw = omw * fs / (2.0 * PI);
+        const double mu = 2595.0 * log10(1.0 + fw / 700.0);
+        const double u = (mu - e0) / delta;
+        int seg;
+        aug::MelBin w;
+        if (!(u >= 0.0)) {
+            seg = -1;
+            w.up = w.down = 0.f;
+        } else if (u >= (double)(M + 1)) {
+            seg = M + 1;
+            w.up = w.down = 0.f;
+        } else {
+            const double fl = floor(u);
+            seg = (int)fl;
+            w.up = (float)(u - fl);
+            w.down = (float)(1.0 - (u - fl));
+        }
+        seg_s[k] = seg;
+        melw[(int64_t)utt * nb + k] = w;
+    }
+    int *st = melstart + (int64_t)utt * (M + 2);
+    for (int m = threadIdx.x; m < M + 2; m += blockDim.x) st[m] = nb;
+    __syncthreads();
+    for (int k = threadIdx.x; k < nb; k += blockDim.x) {
+        const int prev = k ? seg_s[k - 1] : -1;
+        const int cur = seg_s[k];
+        for (int m = prev + 1; m <= cur && m < M + 2; ++m) st[m] = k;   // first bin with seg >= m
+    }
+}
+
+// Filterbank energy of band m for one frame's power spectrum `p`.
+__device__ __forceinline__ float band_energy(const float *p, const aug::MelBin *w, const int *st,
+                                             int m) {
+    float e = 0.f;
+    const int k0 = st[m], k1 = st[m + 1], k2 = st[m + 2];
+    for (int k = k0; k < k1; ++k) e = fmaf(w[k].up, p[k], e);
+    for (int k = k1; k < k2; ++k) e = fmaf(w[k].down, p[k], e);
+    return e;
+}
+
+__device__ __forceinline__ float compress(float e, float floor_v, int mode) {
+    e = fmaxf(e, floor_v);
+    const float l = logf(e);
+    return mode == AUG_COMPRESS_LOG ? l : expf(l * (1.f / 15.f));
+}
+
+// ---------------------------------------------------------------- tile transform
+// Power spectra of `nf` frames starting `hop` apart in `chunk` (shared memory)
+// into ptile[f][k], k <= K/2 (row stride K/2+1).
+template <int K, int E>
+__device__ __forceinline__ void tile_power(const float *chunk, int nf, int win, int hop,
+                                           float2 *fbuf, float *ptile,
+                                           const float2 *__restrict__ tw) {
+    static_assert(K / E == GROUP, "one FFT per 64-thread group");
+    const int tid = threadIdx.x, tg = tid & (GROUP - 1), grp = tid / GROUP;
+    float2 *s = fbuf + grp * K;
+    constexpr int NBP = K / 2 + 1;
+    float wv[E];
+#pragma unroll
+    for (int r = 0; r < E; ++r) {
+        const int n = tg + GROUP * r;
+        wv[r] = n < win ? 0.5f - 0.5f * cospif(2.f * (float)n / (float)win) : 0.f;
+    }
+    const int npair = (nf + 1) / 2;
+    const int iters = (npair + NGROUP - 1) / NGROUP;
+    for (int it = 0; it < iters; ++it) {
+        const int pr = it * NGROUP + grp;
+        const int f0 = 2 * pr;
+        const bool have0 = f0 < nf, have1 = f0 + 1 < nf;
+        float2 v[1][E];
+#pragma unroll
+        for (int r = 0; r < E; ++r) {
+            const int n = tg + GROUP * r;
+            float a = 0.f, b = 0.f;
+            if (n < win) {
+                if (have0) a = wv[r] * chunk[f0 * hop + n];
+                if (have1) b = wv[r] * chunk[(f0 + 1) * hop + n];
+            }
+            v[0][r] = make_float2(a, b);
+        }
+        if constexpr (K == 512) {
+            pass_from_regs<K, E, 8, 1>(v, s, tg, tw);
+            __syncthreads();
+            pass<K, E, 8, 8>(s, tg, tw, CtaSync());
+            pass<K, E, 8, 64>(s, tg, tw, CtaSync());
+        } else {
+            pass_from_regs<K, E, E, 1>(v, s, tg, tw);
+            __syncthreads();
+            pass<K, E, 8, 16>(s, tg, tw, CtaSync());
+            pass<K, E, 8, 128>(s, tg, tw, CtaSync());
+        }
+        if (have0) {
+            float *p0 = ptile + f0 * NBP, *p1 = p0 + NBP;
+            for (int k = tg; k <= K / 2; k += GROUP) {
+                const float2 z = s[k], q = s[(K - k) & (K - 1)];
+                const float ar = z.x + q.x, ai = z.y - q.y;
+                const float br = z.y + q.y, bi = z.x - q.x;
+                p0[k] = 0.25f * (ar * ar + ai * ai);
+                if (have1) p1[k] = 0.25f * (br * br + bi * bi);
+            }
+        }
+        __syncthreads();
+    }
+}
+
+template <int K>
+struct Plan;
+template <>
+struct Plan<512> {
+    static constexpr int E = 8, FT = 32;
+};
+template <>
+struct Plan<1024> {
+    static constexpr int E = 16, FT = 16;
+};
+
+__device__ __forceinline__ float snr_gain_f(const double *energy, int utt, int n_src, float snr_db) {
+    const double es = energy[2 * utt], ev = energy[2 * utt + 1];
+    if (n_src <= 1 || !(es > 0.0) || !(ev > 0.0)) return 0.f;
+    return (float)sqrt(es / (ev * pow(10.0, (double)snr_db / 10.0)));
+}
+
+// MODE 0: wave -> power (global).  MODE 1: y_s + g v -> features.
+template <int K, int MODE>
+__global__ void __launch_bounds__(FEAT_THREADS)
+frames_kernel(const float *__restrict__ in_a, const float *__restrict__ in_b, int64_t in_stride,
+              const double *__restrict__ energy, const AugUttParams *__restrict__ table,
+              const int *__restrict__ lengths, int win, int hop, int M, int T_max,
+              const aug::MelBin *__restrict__ melw, const int *__restrict__ melstart,
+              const float2 *__restrict__ tw, float floor_v, float pad_v, int comp,
+              float *__restrict__ out, int *__restrict__ counts, int n_cap) {
+    constexpr int E = Plan<K>::E, FT = Plan<K>::FT, NBP = K / 2 + 1;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float2 *fbuf = reinterpret_cast<float2 *>(smem_raw);            // [NGROUP][K]
+    float *ptile = reinterpret_cast<float *>(fbuf + NGROUP * K);    // [FT][NBP]
+    float *chunk = ptile + FT * NBP;                                // [(FT-1) hop + win] (+pad)
+    const int chunk_cap = ((FT - 1) * hop + win + 3) & ~3;
+    aug::MelBin *mw = reinterpret_cast<aug::MelBin *>(chunk + chunk_cap);   // [NBP]
+    int *mst = reinterpret_cast<int *>(mw + NBP + 1);                       // [M+2]
+
+    const int utt = blockIdx.y, t0 = blockIdx.x * FT, tid = threadIdx.x;
+    const int N = min(max(lengths[utt], 0), n_cap);
+    const int T = min(frame_count(N, win, hop), T_max);
+    if (blockIdx.x == 0 && tid == 0) counts[utt] = T;
+    const int rows = min(FT, T_max - t0);          // rows of the output this tile owns
+    if (rows <= 0) return;
+    const int nf = max(0, min(FT, T - t0));        // of which real frames
+    const int out_w = MODE == 0 ? NBP : M;
+    float *orow = out + ((int64_t)utt * T_max + t0) * out_w;
+    const float fill = MODE == 0 ? 0.f : pad_v;
+    for (int i = nf * out_w + tid; i < rows * out_w; i += FEAT_THREADS) orow[i] = fill;
+    if (nf == 0) return;
+
+    // stage the samples of these frames
+    const int s0 = t0 * hop;
+    const int ns = (nf - 1) * hop + win;
+    const float *pa = in_a + (int64_t)utt * in_stride + s0;
+    if (MODE == 1) {
+        const float g = snr_gain_f(energy, utt, table[utt].n_src, table[utt].snr_db);
+        const float *pb = in_b + (int64_t)utt * in_stride + s0;
+        if ((hop & 3) == 0) {
+            for (int i = tid * 4; i < ns; i += FEAT_THREADS * 4) {
+                // rows are zero- or garbage-padded up to a multiple of 4 floats but always allocated
+                const float4 x = *reinterpret_cast<const float4 *>(pa + i);
+                float4 y = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (g != 0.f) y = *reinterpret_cast<const float4 *>(pb + i);
+                *reinterpret_cast<float4 *>(chunk + i) = make_float4(
+                    fmaf(g, y.x, x.x), fmaf(g, y.y, x.y), fmaf(g, y.z, x.z), fmaf(g, y.w, x.w));
+            }
+        } else {
+            for (int i = tid; i < ns; i += FEAT_THREADS)
+                chunk[i] = g != 0.f ? fmaf(g, pb[i], pa[i]) : pa[i];
+        }
+        for (int k = tid; k < NBP; k += FEAT_THREADS) mw[k] = melw[(int64_t)utt * NBP + k];
+        for (int m = tid; m < M + 2; m += FEAT_THREADS) mst[m] = melstart[(int64_t)utt * (M + 2) + m];
+    } else {
+        if ((hop & 3) == 0 && (in_stride & 3) == 0) {
+            for (int i = tid * 4; i < ns; i += FEAT_THREADS * 4) {
+                if (s0 + i + 3 < N) {
+                    *reinterpret_cast<float4 *>(chunk + i) = *reinterpret_cast<const float4 *>(pa + i);
+                } else {
+                    for (int j = 0; j < 4; ++j) chunk[i + j] = (s0 + i + j < N) ? pa[i + j] : 0.f;
+                }
+            }
+        } else {
+            for (int i = tid; i < ns; i += FEAT_THREADS) chunk[i] = pa[i];
+        }
+    }
+    __syncthreads();
+
+    tile_power<K, E>(chunk, nf, win, hop, fbuf, ptile, tw);
+
+    if (MODE == 0) {
+        for (int i = tid; i < nf * NBP; i += FEAT_THREADS) orow[i] = ptile[i];
+    } else {
+        for (int i = tid; i < nf * M; i += FEAT_THREADS) {
+            const int f = i / M, m = i - f * M;
+            orow[i] = compress(band_energy(ptile + f * NBP, mw, mst, m), floor_v, comp);
+        }
+    }
+}
+
+// ---------------------------------------------------------------- step 4 alone
+__global__ void __launch_bounds__(256)
+logmel_kernel(const float *__restrict__ power, const int *__restrict__ counts, int NBP, int M,
+              int T_max, const aug::MelBin *__restrict__ melw, const int *__restrict__ melstart,
+              float floor_v, float pad_v, int comp, float *__restrict__ feats) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    aug::MelBin *mw = reinterpret_cast<aug::MelBin *>(smem_raw);
+    int *mst = reinterpret_cast<int *>(mw + NBP + 1);
+    const int utt = blockIdx.y, tid = threadIdx.x;
+    constexpr int FT = 8;
+    const int t0 = blockIdx.x * FT;
+    const int rows = min(FT, T_max - t0);
+    if (rows <= 0) return;
+    const int T = min(max(counts[utt], 0), T_max);
+    for (int k = tid; k < NBP; k += 256) mw[k] = melw[(int64_t)utt * NBP + k];
+    for (int m = tid; m < M + 2; m += 256) mst[m] = melstart[(int64_t)utt * (M + 2) + m];
+    __syncthreads();
+    for (int i = tid; i < rows * M; i += 256) {
+        const int f = i / M, m = i - f * M, t = t0 + f;
+        float val = pad_v;
+        if (t < T)
+            val = compress(band_energy(power + ((int64_t)utt * T_max + t) * NBP, mw, mst, m),
+                           floor_v, comp);
+        feats[((int64_t)utt * T_max + t) * M + m] = val;
+    }
+}
+
+template <int K, int MODE>
+int launch_frames(AugCtx *ctx, const float *a, const float *b, int64_t stride, const int *lengths,
+                  const AugUttParams *table, int B, float *out, int T_max, int *counts) {
+    const AugConfig &c = ctx->cfg;
+    constexpr int FT = Plan<K>::FT, NBP = K / 2 + 1;
+    const int chunk_cap = ((FT - 1) * c.hop + c.win + 3) & ~3;
+    const size_t smem = sizeof(float2) * NGROUP * K + sizeof(float) * FT * NBP +
+                        sizeof(float) * chunk_cap + sizeof(aug::MelBin) * (NBP + 1) +
+                        sizeof(int) * (c.n_mel + 2);
+    if (smem > 227 * 1024) return AUG_ECAP;
+    AUG_CUDA_OK(cudaFuncSetAttribute(frames_kernel<K, MODE>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    dim3 grid((T_max + FT - 1) / FT, B);
+    frames_kernel<K, MODE><<<grid, FEAT_THREADS, smem, ctx->stream>>>(
+        a, b, stride, ctx->energy, table, lengths, c.win, c.hop, c.n_mel, T_max, ctx->melw,
+        ctx->melstart, ctx->tw, c.log_floor, c.pad_value, c.compression, out, counts,
+        (int)(stride < 0x7fffffff ? stride : 0x7fffffff));
+    AUG_CUDA_OK(cudaGetLastError());
+    return AUG_OK;
+}
+
+}  // namespace
+
+int launch_mel_tables(AugCtx *ctx, const AugUttParams *table, int B) {
+    const AugConfig &c = ctx->cfg;
+    mel_tables_kernel<<<B, 256, 0, ctx->stream>>>(table, c.n_fft, c.n_mel, (double)c.fs,
+                                                  (double)c.f_lo, (double)c.f_hi, ctx->melw,
+                                                  ctx->melstart);
+    AUG_CUDA_OK(cudaGetLastError());
+    return AUG_OK;
+}
+
+int launch_stft_power(AugCtx *ctx, const float *wave, int64_t stride, const int *lengths, int B,
+                      float *power, int T_max, int *counts) {
+    if (T_max <= 0) return AUG_OK;
+    if (ctx->cfg.n_fft == 512)
+        return launch_frames<512, 0>(ctx, wave, nullptr, stride, lengths, nullptr, B, power, T_max, counts);
+    return launch_frames<1024, 0>(ctx, wave, nullptr, stride, lengths, nullptr, B, power, T_max, counts);
+}
+
+int launch_fused_features(AugCtx *ctx, const int *lengths, const AugUttParams *table, int B,
+                          float *feats, int T_max, int *counts, float *, int64_t) {
+    if (T_max <= 0) return AUG_OK;
+    if (ctx->cfg.n_fft == 512)
+        return launch_frames<512, 1>(ctx, ctx->ys, ctx->vv, ctx->ws_stride, lengths, table, B, feats,
+                                     T_max, counts);
+    return launch_frames<1024, 1>(ctx, ctx->ys, ctx->vv, ctx->ws_stride, lengths, table, B, feats,
+                                  T_max, counts);
+}
+
+int launch_logmel(AugCtx *ctx, const float *power, const int *counts, int B, int T_max,
+                  float *feats) {
+    const AugConfig &c = ctx->cfg;
+    if (T_max <= 0) return AUG_OK;
+    const int NBP = ctx->n_bins;
+    const size_t smem = sizeof(aug::MelBin) * (NBP + 1) + sizeof(int) * (c.n_mel + 2);
+    dim3 grid((T_max + 7) / 8, B);
+    logmel_kernel<<<grid, 256, smem, ctx->stream>>>(power, counts, NBP, c.n_mel, T_max, ctx->melw,
+                                                    ctx->melstart, c.log_floor, c.pad_value,
+                                                    c.compression, feats);
+    AUG_CUDA_OK(cudaGetLastError());
+    return AUG_OK;
+}

@@ -1,0 +1,154 @@
+// Shared-memory complex FFT building blocks (forward transform, e^{-i...}).
+//
+// A transform of N points is run by N/E threads; each pass keeps E points of a
+// thread in registers as E/R radix-R butterflies and exchanges them through one
+// shared-memory array in Stockham (self-sorting) order, so no bit reversal is
+// needed.  The unnormalised inverse is obtained with the same code by swapping
+// real and imaginary parts on the way in and on the way out.
+#pragma once
+#include <cuda_runtime.h>
+
+namespace augfft {
+
+constexpr int TW_N = 16384;  // the twiddle table holds exp(-2 pi i m / TW_N), m < TW_N
+
+__device__ __forceinline__ float2 cmul(float2 a, float2 b) {
+    return make_float2(fmaf(a.x, b.x, -a.y * b.y), fmaf(a.x, b.y, a.y * b.x));
+}
+__device__ __forceinline__ float2 cadd(float2 a, float2 b) { return make_float2(a.x + b.x, a.y + b.y); }
+__device__ __forceinline__ float2 csub(float2 a, float2 b) { return make_float2(a.x - b.x, a.y - b.y); }
+__device__ __forceinline__ float2 cconj(float2 a) { return make_float2(a.x, -a.y); }
+// a * (-i)
+__device__ __forceinline__ float2 cmul_mi(float2 a) { return make_float2(a.y, -a.x); }
+
+// In-register DFT of R points, natural order in and out.
+template <int R>
+struct Dft;
+
+template <>
+struct Dft<2> {
+    __device__ __forceinline__ static void run(float2 *v) {
+        float2 a = v[0], b = v[1];
+        v[0] = cadd(a, b);
+        v[1] = csub(a, b);
+    }
+};
+
+template <>
+struct Dft<4> {
+    __device__ __forceinline__ static void run(float2 *v) {
+        float2 t0 = cadd(v[0], v[2]), t1 = csub(v[0], v[2]);
+        float2 t2 = cadd(v[1], v[3]), t3 = cmul_mi(csub(v[1], v[3]));
+        v[0] = cadd(t0, t2);
+        v[1] = cadd(t1, t3);
+        v[2] = csub(t0, t2);
+        v[3] = csub(t1, t3);
+    }
+};
+
+template <>
+struct Dft<8> {
+    __device__ __forceinline__ static void run(float2 *v) {
+        const float h = 0.70710678118654752440f;
+        float2 e[4] = {v[0], v[2], v[4], v[6]};
+        float2 o[4] = {v[1], v[3], v[5], v[7]};
+        Dft<4>::run(e);
+        Dft<4>::run(o);
+        // o[k] *= exp(-2 pi i k / 8)
+        o[1] = make_float2(h * (o[1].x + o[1].y), h * (o[1].y - o[1].x));
+        o[2] = cmul_mi(o[2]);
+        o[3] = make_float2(h * (o[3].y - o[3].x), -h * (o[3].x + o[3].y));
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            v[k] = cadd(e[k], o[k]);
+            v[k + 4] = csub(e[k], o[k]);
+        }
+    }
+};
+
+template <>
+struct Dft<16> {
+    __device__ __forceinline__ static void run(float2 *v) {
+        float2 e[8], o[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            e[k] = v[2 * k];
+            o[k] = v[2 * k + 1];
+        }
+        Dft<8>::run(e);
+        Dft<8>::run(o);
+        const float c1 = 0.92387953251128675613f, s1 = 0.38268343236508977173f;
+        const float h = 0.70710678118654752440f;
+        // exp(-2 pi i k / 16), k = 1..7
+        o[1] = cmul(o[1], make_float2(c1, -s1));
+        o[2] = cmul(o[2], make_float2(h, -h));
+        o[3] = cmul(o[3], make_float2(s1, -c1));
+        o[4] = cmul_mi(o[4]);
+        o[5] = cmul(o[5], make_float2(-s1, -c1));
+        o[6] = cmul(o[6], make_float2(-h, -h));
+        o[7] = cmul(o[7], make_float2(-c1, -s1));
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            v[k] = cadd(e[k], o[k]);
+            v[k + 8] = csub(e[k], o[k]);
+        }
+    }
+};
+
+// Multiply v[r] by w^r, r = 1..R-1, with w = exp(-2 pi i k / (NS R)) read from the table.
+template <int R>
+__device__ __forceinline__ void twiddle(float2 *v, float2 w1) {
+    float2 w = w1;
+#pragma unroll
+    for (int r = 1; r < R; ++r) {
+        v[r] = cmul(v[r], w);
+        if (r + 1 < R) w = cmul(w, w1);
+    }
+}
+
+// One pass over registers already holding the inputs of this thread's butterflies:
+//   v[b][r] = data[(t + b T) + r N/R],  T = N/E threads, b < E/R.
+// Applies the pass twiddles (NS = product of earlier radices), the radix-R DFTs,
+// and scatters the results to `s` in Stockham order.  The caller synchronises.
+template <int N, int E, int R, int NS>
+__device__ __forceinline__ void pass_from_regs(float2 (*v)[R], float2 *s, int t,
+                                               const float2 *__restrict__ tw) {
+    constexpr int T = N / E;
+    constexpr int NB = E / R;
+#pragma unroll
+    for (int b = 0; b < NB; ++b) {
+        const int j = t + b * T;
+        const int k = j & (NS - 1);
+        if (NS > 1) {
+            float2 w1 = __ldg(&tw[k * (TW_N / (NS * R))]);
+            twiddle<R>(v[b], w1);
+        }
+        Dft<R>::run(v[b]);
+        const int j0 = (j - k) * R + k;
+#pragma unroll
+        for (int r = 0; r < R; ++r) s[j0 + r * NS] = v[b][r];
+    }
+}
+
+// A full pass: gather from `s`, barrier, transform, scatter, barrier.
+template <int N, int E, int R, int NS, typename Sync>
+__device__ __forceinline__ void pass(float2 *s, int t, const float2 *__restrict__ tw, Sync sync) {
+    constexpr int T = N / E;
+    constexpr int NB = E / R;
+    float2 v[NB][R];
+#pragma unroll
+    for (int b = 0; b < NB; ++b) {
+        const int j = t + b * T;
+#pragma unroll
+        for (int r = 0; r < R; ++r) v[b][r] = s[j + r * (N / R)];
+    }
+    sync();
+    pass_from_regs<N, E, R, NS>(v, s, t, tw);
+    sync();
+}
+
+struct CtaSync {
+    __device__ __forceinline__ void operator()() const { __syncthreads(); }
+};
+
+}  // namespace augfft

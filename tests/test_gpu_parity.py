@@ -1,0 +1,178 @@
+"""GPU parity: every C-ABI entry point against the fp64 CPU checker, element by
+element, on seeded synthetic workloads.  Tolerances (stated once in helpers.py):
+frame counts and padding exact; log-mel within 2e-3 absolute; waveforms within
+1e-4 of the utterance RMS; impulse responses within 2e-5 of their largest tap."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_1912_11040_b200 import binding, synth
+from helpers import (Device, RIR_REL_TOL, check_feats, check_pipeline_against_oracle, check_wave,
+                     oracle_batch)
+
+pytestmark = pytest.mark.gpu
+
+
+def small(index, **kw):
+    return synth.make_workload(index, seed=0, **kw)
+
+
+REDUCED = {
+    1: dict(),                                          # config 1 at full size
+    2: dict(batch=6, dur_scale=0.15),                   # 2 partitions, 1-2 noises, ragged
+    3: dict(batch=3, dur_scale=0.25),                   # 6 partitions, order 20, 3 noises, 80 mel
+    4: dict(batch=12, dur_scale=0.5),                   # many short utterances
+    5: dict(batch=2, dur_scale=0.06),                   # 4 partitions, 1024-point FFT, 128 mel
+}
+
+
+@pytest.mark.parametrize("index", [1, 2, 3, 4, 5])
+def test_rir_matches_image_sum(index):
+    w = small(index, **dict(REDUCED[index], batch=min(REDUCED[index].get("batch", 8), 4),
+                            dur_scale=0.05))
+    dev = Device(w)
+    h = dev.rir().cpu().numpy()
+    for b in range(w.B):
+        row = w.table[b]
+        for s in range(dev.S):
+            if s >= row["n_src"]:
+                assert not h[b, s].any()
+                continue
+            ref = oracle.rir_image_method(row["room"], row["beta"], row["mic"], row["src_pos"][s],
+                                          int(row["order"]), dev.L)
+            err = np.max(np.abs(h[b, s] - ref))
+            assert err <= RIR_REL_TOL * np.max(np.abs(ref)), (index, b, s, err)
+
+
+def test_rir_closed_form_single_image():
+    w = small(1, batch=1, dur_scale=0.05)
+    row = w.table[0]
+    row["room"], row["mic"], row["src_pos"][0] = (50, 8, 4), (2, 3, 1.5), (2 + 42.875, 3, 1.5)
+    row["order"], row["n_src"] = 0, 1
+    dev = Device(w)
+    h = dev.rir().cpu().numpy()[0, 0]
+    assert np.argmax(np.abs(h)) == 2000
+    assert h[2000] == pytest.approx(1 / 42.875, rel=1e-6)
+    h[2000] = 0
+    assert np.max(np.abs(h)) < 1e-8
+
+
+@pytest.mark.parametrize("index", [1, 2, 3, 5])
+def test_reverb_mix_matches_direct_convolution(index):
+    w = small(index, **REDUCED[index]) if index != 1 else small(1, batch=3)
+    dev = Device(w)
+    orc = oracle_batch(w)
+    # feed the CPU impulse responses (rounded to fp32) so this test isolates step 2
+    rir = np.zeros((w.B, dev.S, dev.L), dtype=np.float32)
+    for b, o in orc.items():
+        for s, h in enumerate(o["rirs"]):
+            rir[b, s] = h
+    import torch
+    out = dev.reverb_mix(torch.from_numpy(rir).cuda()).cpu().numpy()
+    for b, o in orc.items():
+        n = int(w.lengths[b])
+        # the reference convolves with the same fp32-rounded impulse responses
+        rirs32 = [rir[b, s].astype(np.float64) for s in range(int(w.table[b]["n_src"]))]
+        noises = [oracle.looped_noise(w.bank, w.table[b]["noise_offset"][k],
+                                      w.table[b]["noise_len"][k], n)
+                  for k in range(int(w.table[b]["n_src"]) - 1)]
+        ref, *_ = oracle.reverb_mix(w.speech[b, :n].astype(np.float64), rirs32, noises,
+                                    w.table[b]["noise_weight"], w.table[b]["snr_db"])
+        check_wave(out[b, :n], ref, f"cfg{index} utt {b}")
+        assert np.all(np.isnan(out[b, n:]))          # samples beyond the length are untouched
+
+
+@pytest.mark.parametrize("index", [1, 5])
+def test_stft_power_and_logmel_match(index):
+    w = small(index, **REDUCED[index]) if index != 1 else small(1, batch=4)
+    w.lengths[0] = 399            # shorter than a window: zero frames
+    w.lengths[1] = 400            # exactly one frame
+    dev = Device(w)
+    P, counts = dev.stft_power(dev.speech)
+    F = dev.logmel(P, counts)
+    P, counts, F = P.cpu().numpy(), counts.cpu().numpy(), F.cpu().numpy()
+    cfg = w.cfg
+    for b in range(w.B):
+        x = w.speech[b, : w.lengths[b]].astype(np.float64)
+        ref = oracle.stft_power(x, cfg["win"], cfg["hop"], cfg["n_fft"])
+        T = ref.shape[0]
+        assert counts[b] == T == oracle.frame_count(len(x), cfg["win"], cfg["hop"])
+        scale = max(ref.max(), 1e-30) if T else 1.0
+        assert np.max(np.abs(P[b, :T] - ref), initial=0.0) <= 2e-6 * scale
+        assert not P[b, T:].any()
+        lm = oracle.logmel(P[b, :T].astype(np.float64), float(w.table[b]["alpha"]), cfg["n_fft"],
+                           cfg["n_mel"])
+        check_feats(F[b, :T], lm, f"utt {b}")
+        assert np.all(F[b, T:] == cfg["pad_value"])
+
+
+@pytest.mark.parametrize("index", [1, 2, 3, 4, 5])
+def test_pipeline_matches_oracle(index):
+    w = small(index, **REDUCED[index])
+    dev = Device(w)
+    F, counts, wave = dev.pipeline(want_wave=True)
+    worst_f, worst_w = check_pipeline_against_oracle(dev, F, counts, wave, oracle_batch(w))
+    print(f"config{index} reduced: worst log-mel err {worst_f:.2e}, worst wave err/rms {worst_w:.2e}")
+
+
+def test_pipeline_edge_lengths_and_no_noise():
+    w = small(2, batch=8, dur_scale=0.12)
+    w.lengths[:6] = [0, 1, 399, 400, 559, 560]
+    for b in range(6):
+        w.speech[b, w.lengths[b]:] = 0
+    w.table["n_src"][6] = 1        # an utterance without noise
+    dev = Device(w)
+    F, counts, wave = dev.pipeline(want_wave=True, lengths_host=False)
+    check_pipeline_against_oracle(dev, F, counts, wave, oracle_batch(w))
+    assert list(counts.cpu().numpy()[:6]) == [0, 0, 0, 1, 1, 2]
+    # identical result when the host lengths are supplied, and without the waveform output
+    F2, counts2, _ = dev.pipeline(want_wave=False, lengths_host=True)
+    assert np.array_equal(counts.cpu().numpy(), counts2.cpu().numpy())
+    assert np.max(np.abs((F - F2).cpu().numpy())) < 1e-3
+
+
+def test_power_law_compression():
+    w = small(1, batch=2)
+    dev = Device(w, compression=binding.COMPRESS_POW_1_15)
+    F, counts, _ = dev.pipeline(want_wave=False)
+    orc = oracle_batch(w, compression="pow15")
+    F = F.cpu().numpy()
+    for b, o in orc.items():
+        T = o["frames"]
+        assert np.max(np.abs(F[b, :T] - o["feats"])) < 2e-3
+
+
+def test_host_buffer_entry_point_matches_device_one():
+    import torch
+    w = small(4, batch=5, dur_scale=0.3)
+    dev = Device(w, host_staging=True)
+    F, counts, _ = dev.pipeline(want_wave=False)
+    Fh = np.full((w.B, dev.T_max, dev.M), np.nan, dtype=np.float32)
+    ch = np.full(w.B, -1, dtype=np.int32)
+    dev.ctx.aug_pipeline_host(w.speech, w.stride, w.lengths, w.bank, w.bank.size,
+                              np.ascontiguousarray(w.table), w.B, Fh, dev.T_max, ch)
+    assert np.array_equal(ch, counts.cpu().numpy())
+    assert np.max(np.abs(Fh - F.cpu().numpy())) < 1e-3
+
+
+def test_errors_and_status_word():
+    w = small(1, batch=2, dur_scale=0.1)
+    dev = Device(w)
+    import torch
+    F = torch.zeros((w.B, dev.T_max, dev.M), device="cuda")
+    c = torch.zeros(w.B, dtype=torch.int32, device="cuda")
+    args = (dev.speech, w.stride, dev.lengths, w.lengths, dev.bank, w.bank.size, dev.table)
+    assert dev.ctx.aug_pipeline(*args, w.B + 1, F, dev.T_max, c, check=False) == binding.AUG_ECAP
+    assert dev.ctx.aug_pipeline(*args, w.B, None, dev.T_max, c, check=False) == binding.AUG_EINVAL
+    assert dev.ctx.aug_pipeline(*args, w.B, F, 1, c, check=False) == binding.AUG_ECAP
+    assert dev.ctx.aug_pipeline(dev.speech, w.stride + 1, *args[2:], w.B, F, dev.T_max, c,
+                                check=False) == binding.AUG_EINVAL
+    # a row the kernels must reject is reported, not faulted on
+    bad = w.table.copy()
+    bad["n_src"][1] = 9
+    tab = binding.table_to_device(bad)
+    rir = torch.zeros((w.B, dev.S, dev.L), device="cuda")
+    dev.ctx.aug_rir_image_method(tab, w.B, rir)
+    assert dev.ctx.aug_last_status() == (1, 1)
+    assert dev.ctx.aug_last_status() == (-1, 0)
+    assert not rir[1].any()
