@@ -1,0 +1,360 @@
+#!/usr/bin/env python
+"""Throughput of the augmentation + feature path: audio-seconds per second.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                  [--workload 1..5]
+
+A step is one aug_pipeline call (impulse responses, partition spectra, filterbank
+tables, convolution + energies, fused mix/STFT/mel/log) over one batch of
+synthetic audio.  `value` is timed with the batch already in HBM; `e2e` times
+aug_pipeline_host, which copies the batch from pinned host memory, runs the path
+and copies features and frame counts back.  With N > 1 every rank runs an
+independent replica of the same job (the path has no exchange step); the ranks
+only meet at the barriers around the timed region.
+
+`--impl reference` times the fp64 CPU checker on bounded samples of the same
+workload on the host cores.
+"""
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "audio-seconds augmented+featurised per second"
+UNIT = "audio-s/s"
+SM_COUNT, FP32_LANES = 148, 128
+
+
+def workload_label(i):
+    return {1: "config1: 8 x 2 s, order 6, 4096 taps, 1 white noise, 40 mel",
+            2: "config2: 256 utts 2-20 s, order 10, 8192 taps, 1-2 noises, 40 mel",
+            3: "config3: 128 x 8 s, order 20, 24000 taps, 3 noises, 80 mel",
+            4: "config4: 4096 utts 1-6 s, order 8, 4096 taps, 1 noise, 40 mel",
+            5: "config5: 64 x 60 s, order 12, 16384 taps, 2 noises, 1024-pt FFT, 128 mel"}[i]
+
+
+# ------------------------------------------------------------------ algorithmic work
+def conv_work(w):
+    """Nominal flops and compulsory bytes of the convolution kernel for one batch:
+    per source one forward real FFT per 4096-sample block (2.5 F log2 F, F = 8192),
+    8 flops per bin and partition for the spectral multiply-accumulate, two inverse
+    FFTs per block; bytes = inputs read once + y_s and v written once + the
+    partition spectra read once."""
+    F, blk = 8192, 4096
+    P = -(-int(w.cfg["rir_taps"]) // blk)
+    fft = 2.5 * F * 13
+    flops = bytes_ = 0.0
+    for b in range(w.B):
+        n, S = int(w.lengths[b]), int(w.table["n_src"][b])
+        nblk = -(-n // blk)
+        flops += nblk * (S * (fft + 8.0 * (F // 2) * P) + (2 if S > 1 else 1) * fft)
+        bytes_ += 4.0 * n * S + 4.0 * n * 2 + S * P * (F // 2) * 8.0
+    return flops, bytes_
+
+
+def feat_work(w):
+    """Fused mix + STFT + mel kernel: one K-point real FFT per frame plus 4 flops per
+    bin; bytes = y_s and v read once + features written once."""
+    K, M = int(w.cfg["n_fft"]), int(w.cfg["n_mel"])
+    flops = bytes_ = 0.0
+    for b in range(w.B):
+        n = int(w.lengths[b])
+        T = 1 + (n - int(w.cfg["win"])) // int(w.cfg["hop"]) if n >= int(w.cfg["win"]) else 0
+        flops += T * (2.5 * K * np.log2(K) + 4.0 * (K // 2 + 1))
+        bytes_ += 8.0 * n + 4.0 * T * M
+    return flops, bytes_
+
+
+# ------------------------------------------------------------------ clocks
+class ClockSampler:
+    def __init__(self, index=0, period=0.02):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thr = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+        self.period = period
+
+    def _run(self):
+        nv = self.nv
+        names = {"hw_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8),
+                 "hw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40),
+                 "sw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20),
+                 "sw_power_cap": getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4)}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for k, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def start(self):
+        if self.nv is not None:
+            self._thr = threading.Thread(target=self._run, daemon=True)
+            self._thr.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thr is not None:
+            self._thr.join()
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------------ CPU checker timing
+def time_oracle(w, budget_s, max_seconds_per_utt=None):
+    """Run the CPU checker over utterances of `w` in order until `budget_s` of wall
+    time is used (at least one).  Returns (audio-s/s, description, cores)."""
+    import oracle
+    oracle._load()
+    cores = os.cpu_count() or 1
+    done_audio = 0.0
+    n_utt = 0
+    t0 = time.perf_counter()
+    for b in range(w.B):
+        n = int(w.lengths[b])
+        if max_seconds_per_utt is not None:
+            n = min(n, int(max_seconds_per_utt * w.cfg["fs"]))
+        oracle.utterance(w.speech[b, :n], w.bank, w.table[b], w.cfg)
+        done_audio += n / w.cfg["fs"]
+        n_utt += 1
+        if time.perf_counter() - t0 >= budget_s:
+            break
+    dt = time.perf_counter() - t0
+    return done_audio / dt, f"first {n_utt} utterance(s), {done_audio:.1f} audio-s, {dt:.1f} s wall", cores
+
+
+def run_reference(args):
+    """The CPU checker as the reference arm: each step is one utterance of the
+    workload (cut to 5 s) through all four steps in fp64 on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    from paper_1912_11040_b200 import synth
+    import oracle
+    oracle._load()
+    w = synth.make_workload(args.workload, seed=0, batch=min(args.steps + args.warmup, 64))
+    cap = int(5.0 * w.cfg["fs"])
+    audio = 0.0
+    times = []
+    for i in range(args.warmup + args.steps):
+        b = i % w.B
+        n = min(int(w.lengths[b]), cap)
+        t0 = time.perf_counter()
+        oracle.utterance(w.speech[b, :n], w.bank, w.table[b], w.cfg)
+        dt = time.perf_counter() - t0
+        if i >= args.warmup:
+            times.append(dt)
+            audio += n / w.cfg["fs"]
+    total = float(sum(times))
+    value = audio / total
+    cores = os.cpu_count() or 1
+    sample = (f"{args.steps} step(s) of one utterance each, cut to 5 s, of {workload_label(args.workload)}; "
+              "direct fp64 convolution, image sum and DFT (OpenMP)")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / max(args.steps, 1),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic",
+            "config": {"workload": workload_label(args.workload), "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+    return 0
+
+
+# ------------------------------------------------------------------ GPU arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_1912_11040_b200 import binding, build, synth
+
+    build.build()
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # every rank runs the same kind of job on its own draw of the workload
+    w = synth.make_workload(args.workload, seed=rank)
+    cfg = binding.make_config(w.cfg, w.B, w.stride, host_staging=True, max_bank_samples=w.bank.size)
+    ctx = binding.AugContext(cfg)
+    speech = torch.from_numpy(w.speech).cuda()
+    lengths = torch.from_numpy(w.lengths).cuda()
+    bank = torch.from_numpy(w.bank).cuda()
+    table = binding.table_to_device(w.table)
+    T_max = binding.aug_frame_count(int(w.lengths.max()), cfg.win, cfg.hop)
+    feats = torch.empty((w.B, T_max, cfg.n_mel), device="cuda")
+    counts = torch.empty(w.B, dtype=torch.int32, device="cuda")
+    rc, bad = binding.aug_validate_params(cfg, w.table, w.bank.size)
+    assert rc == 0, f"table row {bad} invalid"
+
+    def step():
+        ctx.aug_pipeline(speech, w.stride, lengths, w.lengths, bank, w.bank.size, table, w.B,
+                         feats, T_max, counts)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    assert ctx.aug_last_status() == (-1, 0)
+
+    # ---- device-resident timing
+    sampler = ClockSampler(local_rank)
+    ctx.aug_enable_stage_timing(True)
+    launches0 = ctx.aug_launch_count()
+    barrier()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    clocks = sampler.stop()
+    ms_total = e0.elapsed_time(e1)
+    launches = ctx.aug_launch_count() - launches0
+    stage_ms, n_rec = ctx.aug_stage_times()
+    ctx.aug_enable_stage_timing(False)
+
+    # ---- end to end from pinned host buffers
+    sp_h = torch.from_numpy(w.speech).pin_memory()
+    bk_h = torch.from_numpy(w.bank).pin_memory()
+    tb_h = torch.from_numpy(np.ascontiguousarray(w.table).view(np.uint8).reshape(-1).copy()).pin_memory()
+    ln_h = torch.from_numpy(w.lengths).pin_memory()
+    f_h = torch.empty((w.B, T_max, cfg.n_mel)).pin_memory()
+    c_h = torch.empty(w.B, dtype=torch.int32).pin_memory()
+
+    def step_e2e():
+        ctx.aug_pipeline_host(sp_h, w.stride, ln_h, bk_h, w.bank.size, tb_h, w.B, f_h, T_max, c_h)
+
+    e2e_steps = max(3, min(args.steps, 10))
+    for _ in range(2):
+        step_e2e()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        step_e2e()
+    torch.cuda.synchronize()
+    dt_e2e = time.perf_counter() - t0
+    barrier()
+    h2d = sp_h.numel() * 4 + bk_h.numel() * 4 + tb_h.numel() + ln_h.numel() * 4
+    d2h = f_h.numel() * 4 + c_h.numel() * 4
+
+    # ---- reduce over ranks: max time, summed audio
+    audio = torch.tensor([w.audio_seconds, ms_total, dt_e2e], dtype=torch.float64, device="cuda")
+    if world > 1:
+        a = audio.clone()
+        dist.all_reduce(a[0:1], op=dist.ReduceOp.SUM)
+        dist.all_reduce(a[1:3], op=dist.ReduceOp.MAX)
+        audio = a
+    audio_total, ms_total, dt_e2e = (float(v) for v in audio.cpu())
+    value = audio_total * args.steps / (ms_total * 1e-3)
+    e2e_value = audio_total * e2e_steps / dt_e2e
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return 0
+
+    # ---- roofline of the dominant kernel
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except Exception:
+        pass
+    hbm_peak, hbm_src = (peaks["hbm_gbs"], "measured") if "hbm_gbs" in peaks else (6650.0, "fallback")
+    fp32_measured = binding.aug_measure_fp32_peak()
+    fp32_nominal = SM_COUNT * FP32_LANES * 2 * (clocks["sm_max_mhz"] or 1965) * 1e6 / 1e12
+    kernels = {"convolve": (3, conv_work(w)), "features": (5, feat_work(w))}
+    dom = max(kernels, key=lambda k: stage_ms[kernels[k][0]])
+    per_kernel = {}
+    for name, (idx, (flops, byts)) in kernels.items():
+        ms = stage_ms[idx]
+        if ms <= 0:
+            continue
+        t_alu, t_hbm = flops / (fp32_measured * 1e12), byts / (hbm_peak * 1e9)
+        bound = "alu" if t_alu >= t_hbm else "hbm"
+        per_kernel[name] = {
+            "ms": ms, "bound": bound,
+            "tflops": flops / (ms * 1e-3) / 1e12, "frac_fp32": flops / (ms * 1e-3) / 1e12 / fp32_measured,
+            "gbs": byts / (ms * 1e-3) / 1e9, "frac_hbm": byts / (ms * 1e-3) / 1e9 / hbm_peak}
+    d = per_kernel[dom]
+    if d["bound"] == "alu":
+        roofline = {"kernel": dom, "bound": "alu", "achieved": d["tflops"], "peak": fp32_measured,
+                    "unit": "TFLOP/s", "frac": d["frac_fp32"], "traffic": None,
+                    "peak_source": "fp32 FMA loop measured in this run "
+                                   f"(nominal {fp32_nominal:.1f} at max clock)"}
+    else:
+        roofline = {"kernel": dom, "bound": "hbm", "achieved": d["gbs"], "peak": hbm_peak,
+                    "unit": "GB/s", "frac": d["frac_hbm"], "traffic": None,
+                    "peak_source": f"{hbm_src} copy bandwidth"}
+    roofline["per_kernel"] = per_kernel
+    roofline["stage_ms"] = dict(zip(binding.STAGE_NAMES, stage_ms))
+    roofline["stage_calls_averaged"] = n_rec
+
+    cpu_val, cpu_sample, cores = time_oracle(w, args.cpu_budget)
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_total / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic",
+            "config": {"workload": workload_label(args.workload), "batch": w.B,
+                       "audio_seconds_per_step": w.audio_seconds, "parallelism": f"replicas x{world}",
+                       "l2": "inputs larger than L2 (speech + noise bank "
+                             f"{(speech.numel() + bank.numel()) * 4 / 1e6:.0f} MB per step)"},
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+            "gpu_launches": int(launches),
+            "roofline": roofline,
+            "cpu_baseline": {"value": cpu_val, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": cpu_sample}}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", type=int, default=2, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--cpu-budget", type=float, default=15.0,
+                    help="seconds of wall time given to the CPU-checker baseline")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -196,6 +196,28 @@ int aug_pipeline_host(AugCtx *ctx, const float *speech_host, int64_t speech_stri
                       const AugUttParams *table_host, int B, float *feats_host, int T_max,
                       int *frame_counts_host);
 
+/* -------------------------------------------------------------- measurement utilities
+ * (instrumentation of this library; the paper has no counterpart) */
+
+#define AUG_N_STAGES 6 /* 0 impulse responses, 1 partition spectra, 2 filterbank tables,
+                          3 convolution, 4 waveform mix (only when requested), 5 features */
+
+/* on != 0: aug_pipeline records CUDA events between its kernels (up to 256 calls
+ * are kept); on == 0: stop.  Either way the record is cleared. */
+int aug_enable_stage_timing(AugCtx *ctx, int on);
+
+/* Synchronises the stream; ms_host[AUG_N_STAGES] = mean device time of each stage
+ * over the recorded aug_pipeline calls, *n_calls_host = how many; clears the record. */
+int aug_stage_times(AugCtx *ctx, float *ms_host, int *n_calls_host);
+
+/* Kernels this context has launched since aug_create. */
+int64_t aug_launch_count(const AugCtx *ctx);
+
+/* Runs a register-resident FMA loop on every SM of the current device and writes
+ * the best of three fp32 rates (TFLOP/s, 2 flop per FMA) to *tflops_host.
+ * Synchronises cuda_stream. */
+int aug_measure_fp32_peak(void *cuda_stream, float *tflops_host);
+
 #ifdef __cplusplus
 }
 #endif

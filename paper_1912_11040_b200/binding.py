@@ -21,7 +21,10 @@ COMPRESS_LOG, COMPRESS_POW_1_15 = 0, 1
 EXPORTS = ["aug_strerror", "aug_frame_count", "aug_workspace_bytes", "aug_validate_params",
            "aug_create", "aug_destroy", "aug_last_status", "aug_rir_image_method",
            "aug_reverb_mix", "feat_stft_power", "feat_vtlp_logmel", "aug_pipeline",
-           "aug_pipeline_host"]
+           "aug_pipeline_host", "aug_enable_stage_timing", "aug_stage_times", "aug_launch_count",
+           "aug_measure_fp32_peak"]
+N_STAGES = 6
+STAGE_NAMES = ["rir_image", "rir_spectra", "mel_tables", "convolve", "mix", "features"]
 
 
 class AugConfig(ctypes.Structure):
@@ -81,6 +84,14 @@ def lib() -> ctypes.CDLL:
         L.aug_pipeline.argtypes = [vp, vp, i64, vp, vp, vp, i64, vp, i32, vp, i32, vp, vp]
         L.aug_pipeline_host.restype = i32
         L.aug_pipeline_host.argtypes = [vp, vp, i64, vp, vp, i64, vp, i32, vp, i32, vp]
+        L.aug_enable_stage_timing.restype = i32
+        L.aug_enable_stage_timing.argtypes = [vp, i32]
+        L.aug_stage_times.restype = i32
+        L.aug_stage_times.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i32)]
+        L.aug_launch_count.restype = i64
+        L.aug_launch_count.argtypes = [vp]
+        L.aug_measure_fp32_peak.restype = i32
+        L.aug_measure_fp32_peak.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
         _lib = L
     return _lib
 
@@ -117,6 +128,17 @@ def aug_validate_params(config: AugConfig, table: np.ndarray, bank_len: int):
     rc = lib().aug_validate_params(ctypes.byref(config), table.ctypes.data, int(table.shape[0]),
                                    int(bank_len), ctypes.byref(bad))
     return int(rc), int(bad.value)
+
+
+def aug_measure_fp32_peak(stream: Optional[int] = None) -> float:
+    """fp32 FMA rate of the current device in TFLOP/s."""
+    import torch
+    if stream is None:
+        stream = torch.cuda.current_stream().cuda_stream
+    out = ctypes.c_float(0.0)
+    _check(lib().aug_measure_fp32_peak(ctypes.c_void_p(int(stream)), ctypes.byref(out)),
+           "aug_measure_fp32_peak")
+    return float(out.value)
 
 
 def _ptr(t) -> Optional[int]:
@@ -177,6 +199,19 @@ class AugContext:
         _check(lib().aug_last_status(self._h, ctypes.byref(utt), ctypes.byref(why)),
                "aug_last_status")
         return int(utt.value), int(why.value)
+
+    def aug_enable_stage_timing(self, on: bool):
+        _check(lib().aug_enable_stage_timing(self._h, int(bool(on))), "aug_enable_stage_timing")
+
+    def aug_stage_times(self):
+        """(mean ms per stage, number of aug_pipeline calls averaged)."""
+        ms = (ctypes.c_float * N_STAGES)()
+        n = ctypes.c_int(0)
+        _check(lib().aug_stage_times(self._h, ms, ctypes.byref(n)), "aug_stage_times")
+        return [float(v) for v in ms], int(n.value)
+
+    def aug_launch_count(self) -> int:
+        return int(lib().aug_launch_count(self._h))
 
     def aug_rir_image_method(self, table_dev, B, rir_dev, check=True):
         return self._ret(lib().aug_rir_image_method(self._h, _ptr(table_dev), int(B),

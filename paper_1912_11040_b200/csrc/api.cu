@@ -210,6 +210,10 @@ int aug_destroy(AugCtx *ctx) {
     if (!ctx) return AUG_OK;
     int rc = AUG_OK;
     if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) rc = AUG_ECUDA;
+    if (ctx->ev) {
+        for (int i = 0; i < aug::EV_RING * (AUG_N_STAGES + 1); ++i) cudaEventDestroy(ctx->ev[i]);
+        free(ctx->ev);
+    }
     if (cudaFree(ctx->ws_base) != cudaSuccess) rc = AUG_ECUDA;
     delete ctx;
     return rc;
@@ -299,16 +303,29 @@ int aug_pipeline(AugCtx *ctx, const float *speech_dev, int64_t speech_stride,
         if (aug_frame_count(mx, ctx->cfg.win, ctx->cfg.hop) > T_max) return AUG_ECAP;
         max_len = mx;
     }
+    cudaEvent_t *ev = nullptr;
+    if (ctx->timing && ctx->ev && ctx->ev_n < aug::EV_RING)
+        ev = ctx->ev + (size_t)ctx->ev_n * (AUG_N_STAGES + 1);
+    auto mark = [&](int i) { if (ev) cudaEventRecord(ev[i], ctx->stream); };
+    mark(0);
     if ((rc = launch_rir(ctx, table_dev, B, ctx->rir)) != AUG_OK) return rc;
+    mark(1);
     if ((rc = launch_rir_spectra(ctx, ctx->rir, table_dev, B)) != AUG_OK) return rc;
+    mark(2);
     if ((rc = launch_mel_tables(ctx, table_dev, B)) != AUG_OK) return rc;
+    mark(3);
     if ((rc = launch_convolve(ctx, speech_dev, speech_stride, lengths_dev, noise_bank_dev, bank_len,
                               table_dev, B, max_len)) != AUG_OK) return rc;
+    mark(4);
     if (wave_out &&
         (rc = launch_mix(ctx, lengths_dev, table_dev, B, max_len, wave_out, speech_stride)) != AUG_OK)
         return rc;
-    return launch_fused_features(ctx, lengths_dev, table_dev, B, feats_dev, T_max, frame_counts_dev,
-                                 nullptr, 0);
+    mark(5);
+    rc = launch_fused_features(ctx, lengths_dev, table_dev, B, feats_dev, T_max, frame_counts_dev,
+                               nullptr, 0);
+    mark(6);
+    if (ev && rc == AUG_OK) ctx->ev_n++;
+    return rc;
 }
 
 int aug_pipeline_host(AugCtx *ctx, const float *speech_host, int64_t speech_stride,
@@ -346,5 +363,46 @@ int aug_pipeline_host(AugCtx *ctx, const float *speech_host, int64_t speech_stri
     AUG_CUDA_OK(cudaStreamSynchronize(st));
     return AUG_OK;
 }
+
+int aug_enable_stage_timing(AugCtx *ctx, int on) {
+    if (!ctx) return AUG_EINVAL;
+    AUG_CUDA_OK(cudaStreamSynchronize(ctx->stream));
+    if (on && !ctx->ev) {
+        const int n = aug::EV_RING * (AUG_N_STAGES + 1);
+        ctx->ev = static_cast<cudaEvent_t *>(calloc(n, sizeof(cudaEvent_t)));
+        if (!ctx->ev) return AUG_ENOMEM;
+        for (int i = 0; i < n; ++i) {
+            if (cudaEventCreate(&ctx->ev[i]) != cudaSuccess) {
+                for (int j = 0; j < i; ++j) cudaEventDestroy(ctx->ev[j]);
+                free(ctx->ev);
+                ctx->ev = nullptr;
+                return AUG_ECUDA;
+            }
+        }
+    }
+    ctx->timing = on ? 1 : 0;
+    ctx->ev_n = 0;
+    return AUG_OK;
+}
+
+int aug_stage_times(AugCtx *ctx, float *ms_host, int *n_calls_host) {
+    if (!ctx || !ms_host) return AUG_EINVAL;
+    AUG_CUDA_OK(cudaStreamSynchronize(ctx->stream));
+    double acc[AUG_N_STAGES] = {0};
+    for (int c = 0; c < ctx->ev_n; ++c) {
+        cudaEvent_t *ev = ctx->ev + (size_t)c * (AUG_N_STAGES + 1);
+        for (int i = 0; i < AUG_N_STAGES; ++i) {
+            float ms = 0.f;
+            AUG_CUDA_OK(cudaEventElapsedTime(&ms, ev[i], ev[i + 1]));
+            acc[i] += ms;
+        }
+    }
+    for (int i = 0; i < AUG_N_STAGES; ++i) ms_host[i] = ctx->ev_n ? (float)(acc[i] / ctx->ev_n) : 0.f;
+    if (n_calls_host) *n_calls_host = ctx->ev_n;
+    ctx->ev_n = 0;
+    return AUG_OK;
+}
+
+int64_t aug_launch_count(const AugCtx *ctx) { return ctx ? ctx->launches : 0; }
 
 }  // extern "C"

@@ -15,6 +15,8 @@ constexpr int MAX_ORDER = 32;
 constexpr int MAX_HALF_W = 47;
 constexpr int MAX_MEL = 128;
 
+constexpr int EV_RING = 256;
+
 enum Reason { R_NONE = 0, R_NSRC = 1, R_ORDER = 2, R_NOISE = 3, R_WAIT = 4 };
 
 // Per-bin entry of the warped filterbank: the bin lies in edge interval `seg`
@@ -47,6 +49,11 @@ struct AugCtx {
     int *melstart;         // [max_batch][n_mel + 2]
     int *status;           // [2]: utterance, reason
     int *counts_tmp;       // [max_batch]
+    // instrumentation
+    int64_t launches;      // kernels launched so far
+    int timing;            // record events between the stages of aug_pipeline
+    cudaEvent_t *ev;       // [EV_RING][AUG_N_STAGES + 1]
+    int ev_n;              // calls recorded
     // staging for the host-buffer entry point (NULL unless cfg.host_staging)
     float *st_speech;      // [max_batch][ws_stride]
     float *st_bank;        // [max_bank_samples]

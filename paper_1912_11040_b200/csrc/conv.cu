@@ -296,6 +296,7 @@ int launch_rir_spectra(AugCtx *ctx, const float *rir, const AugUttParams *table,
     rir_spectra_kernel<<<grid, CT, smem, ctx->stream>>>(rir, table, c.max_sources, c.rir_taps,
                                                         ctx->n_part, ctx->tw, ctx->hspec);
     AUG_CUDA_OK(cudaGetLastError());
+    ctx->launches++;
     return AUG_OK;
 }
 
@@ -314,6 +315,7 @@ int launch_convolve(AugCtx *ctx, const float *speech, int64_t stride, const int 
                                                      ctx->ys, ctx->vv, ctx->ws_stride, ctx->energy,
                                                      ctx->status, max_len);
     AUG_CUDA_OK(cudaGetLastError());
+    ctx->launches++;
     return AUG_OK;
 }
 
@@ -324,5 +326,6 @@ int launch_mix(AugCtx *ctx, const int *lengths, const AugUttParams *table, int B
     mix_kernel<<<grid, 256, 0, ctx->stream>>>(ctx->ys, ctx->vv, ctx->ws_stride, ctx->energy, lengths,
                                               table, wave_out, out_stride, max_len);
     AUG_CUDA_OK(cudaGetLastError());
+    ctx->launches++;
     return AUG_OK;
 }

@@ -289,6 +289,7 @@ int launch_frames(AugCtx *ctx, const float *a, const float *b, int64_t stride, c
         ctx->melstart, ctx->tw, c.log_floor, c.pad_value, c.compression, out, counts,
         (int)(stride < 0x7fffffff ? stride : 0x7fffffff));
     AUG_CUDA_OK(cudaGetLastError());
+    ctx->launches++;
     return AUG_OK;
 }
 
@@ -300,6 +301,7 @@ int launch_mel_tables(AugCtx *ctx, const AugUttParams *table, int B) {
                                                   (double)c.f_lo, (double)c.f_hi, ctx->melw,
                                                   ctx->melstart);
     AUG_CUDA_OK(cudaGetLastError());
+    ctx->launches++;
     return AUG_OK;
 }
 
@@ -332,5 +334,6 @@ int launch_logmel(AugCtx *ctx, const float *power, const int *counts, int B, int
                                                     ctx->melstart, c.log_floor, c.pad_value,
                                                     c.compression, feats);
     AUG_CUDA_OK(cudaGetLastError());
+    ctx->launches++;
     return AUG_OK;
 }

@@ -96,14 +96,19 @@ struct Dft<16> {
 };
 
 // Multiply v[r] by w^r, r = 1..R-1, with w = exp(-2 pi i k / (NS R)) read from the table.
+// Powers are built by squaring (w^2, w^4, w^8) and one more product each, so no
+// power is more than three roundings away from the table value.
 template <int R>
 __device__ __forceinline__ void twiddle(float2 *v, float2 w1) {
-    float2 w = w1;
+    float2 w[R];
+    w[1] = w1;
 #pragma unroll
-    for (int r = 1; r < R; ++r) {
-        v[r] = cmul(v[r], w);
-        if (r + 1 < R) w = cmul(w, w1);
+    for (int r = 2; r < R; ++r) {
+        const int hi = (r & (r - 1)) ? (r & -r) : r / 2;   // split r = hi + lo with hi a power of two
+        w[r] = cmul(w[hi], w[r - hi]);
     }
+#pragma unroll
+    for (int r = 1; r < R; ++r) v[r] = cmul(v[r], w[r]);
 }
 
 // One pass over registers already holding the inputs of this thread's butterflies:

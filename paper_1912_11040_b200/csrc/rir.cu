@@ -139,5 +139,6 @@ int launch_rir(AugCtx *ctx, const AugUttParams *table, int B, float *rir) {
         table, c.max_sources, c.rir_taps, c.frac_half_width, (double)c.fs, (double)c.sound_speed,
         c.max_order, rir, ctx->status);
     AUG_CUDA_OK(cudaGetLastError());
+    ctx->launches++;
     return AUG_OK;
 }
