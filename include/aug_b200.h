@@ -176,6 +176,40 @@ int feat_stft_power(AugCtx *ctx, const float *wave_dev, int64_t stride, const in
 int feat_vtlp_logmel(AugCtx *ctx, const float *power_dev, const int *frame_counts_dev,
                      const AugUttParams *table_dev, int B, int T_max, float *feats_dev);
 
+/* -------------------------------------------------------------- step 4, allocation-free
+ * (an addition of this library; the paper has no counterpart)
+ *
+ * The same computation as feat_vtlp_logmel for callers that cannot allocate
+ * device memory and therefore cannot own an AugCtx (aug_create calls cudaMalloc):
+ * code embedded in an application whose memory pool already holds the whole
+ * device, latency-critical front-ends that must stay off the allocator once
+ * running, or components that are only ever handed device pointers and a stream.
+ * The per-utterance filterbank tables the kernels need are kept in a fixed array
+ * built into the library (about 1.13 MiB; every GPU that loads the library holds
+ * it until the process exits).  This call and everything it calls performs no
+ * cudaMalloc / cudaFree and uses no allocating library.
+ *
+ *   cfg_host     only n_fft, n_mel, fs, f_lo, f_hi, log_floor, pad_value and
+ *                compression are read
+ *   power_dev, frame_counts_dev, table_dev, feats_dev, T_max: as feat_vtlp_logmel
+ *   cuda_stream  cudaStream_t to enqueue on (NULL = default stream); returns
+ *                without synchronising
+ *
+ * Limits: B <= AUG_NOALLOC_MAX_BATCH and n_mel <= 128, else AUG_ECAP ("request
+ * exceeds the capacity ..."); n_fft must be 512 or 1024, else AUG_EINVAL.  Larger
+ * batches must be split by the caller.
+ * First call on a device: it looks up the device address of the built-in array
+ * (cudaGetSymbolAddress, once per device, with that device current).  Make that
+ * first call during start-up, before any stream capture is begun.
+ * Sharing: all calls in the process use the one array on a device and it keeps
+ * whatever the last call wrote.  Each call rewrites the part it reads, so stale
+ * contents are never used, but two calls that can run at the same time on the
+ * GPU (different streams, different host threads) race on it: serialise them. */
+#define AUG_NOALLOC_MAX_BATCH 256
+int feat_vtlp_logmel_noalloc(const AugConfig *cfg_host, const float *power_dev,
+                             const int *frame_counts_dev, const AugUttParams *table_dev, int B,
+                             int T_max, float *feats_dev, void *cuda_stream);
+
 /* -------------------------------------------------------------- steps 1-4
  * The whole path for a batch.  Arguments as above; additionally
  *   lengths_host  the same lengths in host memory (may be NULL): used only to size

@@ -22,7 +22,8 @@ EXPORTS = ["aug_strerror", "aug_frame_count", "aug_workspace_bytes", "aug_valida
            "aug_create", "aug_destroy", "aug_last_status", "aug_rir_image_method",
            "aug_reverb_mix", "feat_stft_power", "feat_vtlp_logmel", "aug_pipeline",
            "aug_pipeline_host", "aug_enable_stage_timing", "aug_stage_times", "aug_launch_count",
-           "aug_measure_fp32_peak"]
+           "aug_measure_fp32_peak", "feat_vtlp_logmel_noalloc"]
+NOALLOC_MAX_BATCH = 256
 N_STAGES = 6
 STAGE_NAMES = ["rir_image", "rir_spectra", "mel_tables", "convolve", "mix", "features"]
 
@@ -84,6 +85,8 @@ def lib() -> ctypes.CDLL:
         L.aug_pipeline.argtypes = [vp, vp, i64, vp, vp, vp, i64, vp, i32, vp, i32, vp, vp]
         L.aug_pipeline_host.restype = i32
         L.aug_pipeline_host.argtypes = [vp, vp, i64, vp, vp, i64, vp, i32, vp, i32, vp]
+        L.feat_vtlp_logmel_noalloc.restype = i32
+        L.feat_vtlp_logmel_noalloc.argtypes = [ctypes.POINTER(AugConfig), vp, vp, vp, i32, i32, vp, vp]
         L.aug_enable_stage_timing.restype = i32
         L.aug_enable_stage_timing.argtypes = [vp, i32]
         L.aug_stage_times.restype = i32
@@ -139,6 +142,25 @@ def aug_measure_fp32_peak(stream: Optional[int] = None) -> float:
     _check(lib().aug_measure_fp32_peak(ctypes.c_void_p(int(stream)), ctypes.byref(out)),
            "aug_measure_fp32_peak")
     return float(out.value)
+
+
+def feat_vtlp_logmel_noalloc(config: AugConfig, power_dev, counts_dev, table_dev, B: int,
+                             T_max: int, feats_dev, stream: Optional[int] = None,
+                             check: bool = True) -> int:
+    """Step 4 for callers that may not allocate device memory: no context, the
+    filterbank tables live in an array built into the library (at most
+    NOALLOC_MAX_BATCH utterances per call).  Enqueues on `stream` (default: torch's
+    current stream) and returns the status code; raises AugError when `check`."""
+    if stream is None:
+        import torch
+        stream = torch.cuda.current_stream().cuda_stream
+    rc = int(lib().feat_vtlp_logmel_noalloc(ctypes.byref(config), _ptr(power_dev),
+                                            _ptr(counts_dev), _ptr(table_dev), int(B),
+                                            int(T_max), _ptr(feats_dev),
+                                            ctypes.c_void_p(int(stream))))
+    if check:
+        _check(rc, "feat_vtlp_logmel_noalloc")
+    return rc
 
 
 def _ptr(t) -> Optional[int]:

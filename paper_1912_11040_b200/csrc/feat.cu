@@ -337,3 +337,89 @@ int launch_logmel(AugCtx *ctx, const float *power, const int *counts, int B, int
     ctx->launches++;
     return AUG_OK;
 }
+
+// ---------------------------------------------------------------- step 4 without any allocation
+//
+// feat_vtlp_logmel needs two small per-utterance tables (filterbank weights per
+// DFT bin, first bin of every band interval) that normally live in the context's
+// workspace, and a context cannot exist without cudaMalloc.  Some callers are not
+// allowed to allocate: a plug-in running inside a host application that has
+// handed every byte of device memory to its own pool, a real-time feature
+// front-end that must not touch the allocator after start-up, or code that only
+// receives device pointers and a stream.  For them the tables live in a
+// fixed-size array that is part of the loaded library image, so nothing is
+// allocated at call time -- at the price that every GPU that loads the library
+// carries the array until the process exits, and that all calls share it.
+namespace {
+
+constexpr int NOALLOC_BINS = 513;                                   // n_fft <= 1024
+constexpr size_t NOALLOC_MELW_BYTES =
+    sizeof(aug::MelBin) * (size_t)AUG_NOALLOC_MAX_BATCH * NOALLOC_BINS;          // 1 050 624
+constexpr size_t NOALLOC_START_BYTES =
+    sizeof(int) * (size_t)AUG_NOALLOC_MAX_BATCH * (aug::MAX_MEL + 2);            //   133 120
+static_assert(NOALLOC_MELW_BYTES % 256 == 0, "second table must stay 256-byte aligned");
+
+// The scratch itself.  In host code this name is only a handle for the runtime,
+// not an address a kernel could use; the device address is looked up below.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[NOALLOC_MELW_BYTES + NOALLOC_START_BYTES];
+
+constexpr int NOALLOC_MAX_DEVICES = 64;
+void *g_noalloc_addr[NOALLOC_MAX_DEVICES];   // device address of the scratch, per device; NULL = not looked up yet
+
+// Device address of the scratch on the current device.  The first call on a
+// device asks the runtime for it (no allocation: the array already exists in the
+// module); later calls reuse the cached pointer.
+int noalloc_scratch(void **out) {
+    int dev = -1;
+    AUG_CUDA_OK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= NOALLOC_MAX_DEVICES) return AUG_ECAP;
+    void *p = __atomic_load_n(&g_noalloc_addr[dev], __ATOMIC_ACQUIRE);
+    if (!p) {
+        AUG_CUDA_OK(cudaGetSymbolAddress(&p, g_noalloc_scratch));
+        if (!p) return AUG_ECUDA;
+        __atomic_store_n(&g_noalloc_addr[dev], p, __ATOMIC_RELEASE);   // same value from any thread
+    }
+    *out = p;
+    return AUG_OK;
+}
+
+}  // namespace
+
+extern "C" int feat_vtlp_logmel_noalloc(const AugConfig *cfg, const float *power_dev,
+                                        const int *frame_counts_dev,
+                                        const AugUttParams *table_dev, int B, int T_max,
+                                        float *feats_dev, void *cuda_stream) {
+    if (!cfg || !power_dev || !frame_counts_dev || !table_dev || !feats_dev) return AUG_EINVAL;
+    if (B < 0 || T_max <= 0) return AUG_EINVAL;
+    if (cfg->n_fft != 512 && cfg->n_fft != 1024) return AUG_EINVAL;
+    if (cfg->n_mel < 1 || cfg->fs <= 0 || !(cfg->f_lo >= 0.f) || !(cfg->f_hi > cfg->f_lo) ||
+        !(cfg->log_floor > 0.f))
+        return AUG_EINVAL;
+    if (cfg->compression != AUG_COMPRESS_LOG && cfg->compression != AUG_COMPRESS_POW_1_15)
+        return AUG_EINVAL;
+    // the fixed scratch holds tables for this many utterances and bands, no more
+    if (B > AUG_NOALLOC_MAX_BATCH || cfg->n_mel > aug::MAX_MEL) return AUG_ECAP;
+    if (B == 0) return AUG_OK;
+
+    void *scratch = nullptr;
+    int rc = noalloc_scratch(&scratch);
+    if (rc != AUG_OK) return rc;
+    aug::MelBin *melw = reinterpret_cast<aug::MelBin *>(scratch);
+    int *melstart = reinterpret_cast<int *>(static_cast<unsigned char *>(scratch) + NOALLOC_MELW_BYTES);
+
+    // Both tables are written in full for utterances [0, B) before they are read
+    // (same stream), so nothing left by an earlier call is ever seen and nothing
+    // needs clearing.
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const int nbp = cfg->n_fft / 2 + 1;
+    mel_tables_kernel<<<B, 256, 0, st>>>(table_dev, cfg->n_fft, cfg->n_mel, (double)cfg->fs,
+                                         (double)cfg->f_lo, (double)cfg->f_hi, melw, melstart);
+    AUG_CUDA_OK(cudaGetLastError());
+    const size_t smem = sizeof(aug::MelBin) * (nbp + 1) + sizeof(int) * (cfg->n_mel + 2);
+    dim3 grid((T_max + 7) / 8, B);
+    logmel_kernel<<<grid, 256, smem, st>>>(power_dev, frame_counts_dev, nbp, cfg->n_mel, T_max,
+                                           melw, melstart, cfg->log_floor, cfg->pad_value,
+                                           cfg->compression, feats_dev);
+    AUG_CUDA_OK(cudaGetLastError());
+    return AUG_OK;
+}
