@@ -203,7 +203,7 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     # every rank runs the same kind of job on its own draw of the workload
-    w = synth.make_workload(args.workload, seed=rank)
+    w = synth.make_workload(args.workload, seed=rank, batch=args.batch)
     cfg = binding.make_config(w.cfg, w.B, w.stride, host_staging=True, max_bank_samples=w.bank.size)
     ctx = binding.AugContext(cfg)
     speech = torch.from_numpy(w.speech).cuda()
@@ -254,8 +254,8 @@ def run_ours(args):
     def step_e2e():
         ctx.aug_pipeline_host(sp_h, w.stride, ln_h, bk_h, w.bank.size, tb_h, w.B, f_h, T_max, c_h)
 
-    e2e_steps = max(3, min(args.steps, 10))
-    for _ in range(2):
+    e2e_steps = 1 if args.skip_e2e else max(3, min(args.steps, 10))
+    for _ in range(0 if args.skip_e2e else 2):
         step_e2e()
     barrier()
     t0 = time.perf_counter()
@@ -319,7 +319,10 @@ def run_ours(args):
     roofline["stage_ms"] = dict(zip(binding.STAGE_NAMES, stage_ms))
     roofline["stage_calls_averaged"] = n_rec
 
-    cpu_val, cpu_sample, cores = time_oracle(w, args.cpu_budget)
+    if args.cpu_budget > 0:
+        cpu_val, cpu_sample, cores = time_oracle(w, args.cpu_budget)
+    else:
+        cpu_val, cpu_sample, cores = None, "skipped (--cpu-budget 0)", os.cpu_count() or 1
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_total / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
@@ -350,6 +353,10 @@ def main():
     ap.add_argument("--workload", type=int, default=2, choices=[1, 2, 3, 4, 5])
     ap.add_argument("--cpu-budget", type=float, default=15.0,
                     help="seconds of wall time given to the CPU-checker baseline")
+    ap.add_argument("--batch", type=int, default=None,
+                    help="profiling runs: fewer utterances than the workload's own batch")
+    ap.add_argument("--skip-e2e", action="store_true",
+                    help="profiling runs: one end-to-end step instead of a timed series")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)

@@ -32,8 +32,9 @@ int check_config(const AugConfig *c) {
 }
 
 struct Layout {
-    int n_part, n_bins, t_cap;
+    int n_part, n_bins, t_cap, nblk_cap;
     int64_t ws_stride;
+    int64_t off_xspec;
     int64_t off_tw, off_rir, off_hspec, off_ys, off_vv, off_energy, off_melw, off_melstart,
         off_status, off_counts, off_st_speech, off_st_bank, off_st_table, off_st_lengths,
         off_st_feats, off_st_counts, total;
@@ -51,6 +52,8 @@ Layout make_layout(const AugConfig &c) {
     l.off_tw = take(sizeof(float2) * augfft::TW_N);
     l.off_rir = take(sizeof(float) * B * S * c.rir_taps);
     l.off_hspec = take(sizeof(float2) * B * S * l.n_part * aug::CONV_N2);
+    l.nblk_cap = (c.max_samples + aug::CONV_BLK - 1) / aug::CONV_BLK;
+    l.off_xspec = l.n_part > 1 ? take(sizeof(float2) * B * S * l.nblk_cap * aug::CONV_N2) : -1;
     l.off_ys = take(sizeof(float) * B * l.ws_stride);
     l.off_vv = take(sizeof(float) * B * l.ws_stride);
     l.off_energy = take(sizeof(double) * 2 * B);
@@ -170,6 +173,8 @@ int aug_create(AugCtx **out, const AugConfig *cfg, void *cuda_stream) {
     ctx->tw = reinterpret_cast<float2 *>(base + l.off_tw);
     ctx->rir = reinterpret_cast<float *>(base + l.off_rir);
     ctx->hspec = reinterpret_cast<float2 *>(base + l.off_hspec);
+    ctx->nblk_cap = l.nblk_cap;
+    ctx->xspec = l.off_xspec >= 0 ? reinterpret_cast<float2 *>(base + l.off_xspec) : nullptr;
     ctx->ys = reinterpret_cast<float *>(base + l.off_ys);
     ctx->vv = reinterpret_cast<float *>(base + l.off_vv);
     ctx->energy = reinterpret_cast<double *>(base + l.off_energy);

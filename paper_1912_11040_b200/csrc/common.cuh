@@ -42,6 +42,8 @@ struct AugCtx {
     float2 *tw;            // [TW_N] twiddles
     float *rir;            // [max_batch][max_sources][rir_taps]
     float2 *hspec;         // [max_batch][max_sources][n_part][CONV_N2]
+    float2 *xspec;         // [max_batch][max_sources][nblk_cap][CONV_N2]; NULL when n_part == 1
+    int nblk_cap;          // blocks of an utterance of max_samples
     float *ys;             // [max_batch][ws_stride]
     float *vv;             // [max_batch][ws_stride]
     double *energy;        // [max_batch][2]

@@ -97,7 +97,7 @@ __device__ __forceinline__ void tile_power(const float *chunk, int nf, int win, 
                                            const float2 *__restrict__ tw) {
     static_assert(K / E == GROUP, "one FFT per 64-thread group");
     const int tid = threadIdx.x, tg = tid & (GROUP - 1), grp = tid / GROUP;
-    float2 *s = fbuf + grp * K;
+    float2 *s = fbuf + grp * padded_points(K);
     constexpr int NBP = K / 2 + 1;
     float wv[E];
 #pragma unroll
@@ -125,18 +125,18 @@ __device__ __forceinline__ void tile_power(const float *chunk, int nf, int win, 
         if constexpr (K == 512) {
             pass_from_regs<K, E, 8, 1>(v, s, tg, tw);
             __syncthreads();
-            pass<K, E, 8, 8>(s, tg, tw, CtaSync());
-            pass<K, E, 8, 64>(s, tg, tw, CtaSync());
+            pass<K, E, 8, 8, 1>(s, tg, tw, CtaSync());
+            pass<K, E, 8, 64, 8>(s, tg, tw, CtaSync());
         } else {
             pass_from_regs<K, E, E, 1>(v, s, tg, tw);
             __syncthreads();
-            pass<K, E, 8, 16>(s, tg, tw, CtaSync());
-            pass<K, E, 8, 128>(s, tg, tw, CtaSync());
+            pass<K, E, 8, 16, 1>(s, tg, tw, CtaSync());
+            pass<K, E, 8, 128, 16>(s, tg, tw, CtaSync());
         }
         if (have0) {
             float *p0 = ptile + f0 * NBP, *p1 = p0 + NBP;
             for (int k = tg; k <= K / 2; k += GROUP) {
-                const float2 z = s[k], q = s[(K - k) & (K - 1)];
+                const float2 z = s[pad0(k)], q = s[pad0((K - k) & (K - 1))];
                 const float ar = z.x + q.x, ai = z.y - q.y;
                 const float br = z.y + q.y, bi = z.x - q.x;
                 p0[k] = 0.25f * (ar * ar + ai * ai);
@@ -175,8 +175,8 @@ frames_kernel(const float *__restrict__ in_a, const float *__restrict__ in_b, in
               float *__restrict__ out, int *__restrict__ counts, int n_cap) {
     constexpr int E = Plan<K>::E, FT = Plan<K>::FT, NBP = K / 2 + 1;
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    float2 *fbuf = reinterpret_cast<float2 *>(smem_raw);            // [NGROUP][K]
-    float *ptile = reinterpret_cast<float *>(fbuf + NGROUP * K);    // [FT][NBP]
+    float2 *fbuf = reinterpret_cast<float2 *>(smem_raw);            // [NGROUP][K + K/8]
+    float *ptile = reinterpret_cast<float *>(fbuf + NGROUP * padded_points(K));    // [FT][NBP]
     float *chunk = ptile + FT * NBP;                                // [(FT-1) hop + win] (+pad)
     const int chunk_cap = ((FT - 1) * hop + win + 3) & ~3;
     aug::MelBin *mw = reinterpret_cast<aug::MelBin *>(chunk + chunk_cap);   // [NBP]
@@ -277,7 +277,7 @@ int launch_frames(AugCtx *ctx, const float *a, const float *b, int64_t stride, c
     const AugConfig &c = ctx->cfg;
     constexpr int FT = Plan<K>::FT, NBP = K / 2 + 1;
     const int chunk_cap = ((FT - 1) * c.hop + c.win + 3) & ~3;
-    const size_t smem = sizeof(float2) * NGROUP * K + sizeof(float) * FT * NBP +
+    const size_t smem = sizeof(float2) * NGROUP * padded_points(K) + sizeof(float) * FT * NBP +
                         sizeof(float) * chunk_cap + sizeof(aug::MelBin) * (NBP + 1) +
                         sizeof(int) * (c.n_mel + 2);
     if (smem > 227 * 1024) return AUG_ECAP;

@@ -101,6 +101,7 @@ struct Dft<16> {
 template <int R>
 __device__ __forceinline__ void twiddle(float2 *v, float2 w1) {
     float2 w[R];
+    w[0] = make_float2(1.f, 0.f);
     w[1] = w1;
 #pragma unroll
     for (int r = 2; r < R; ++r) {
@@ -111,6 +112,19 @@ __device__ __forceinline__ void twiddle(float2 *v, float2 w1) {
     for (int r = 1; r < R; ++r) v[r] = cmul(v[r], w[r]);
 }
 
+// Shared-memory index padding.  Complex points are 8 bytes, 16 of them span the 32
+// banks; element i lives at i + ((i >> 4) << PS), i.e. every row of 16 points is
+// shifted by 1 (PS = 0) or 2 (PS = 1) slots per row.  Row-constant shifts keep the
+// unit-stride gathers conflict-free; the shift is chosen per pass so that its
+// scatter is conflict-free too: stride-R scatters (NS = 1) want 1 per row, the
+// NS = 8 scatter (rows 4 apart within a half-warp) wants 2 per row.
+template <int PS>
+__device__ __forceinline__ int padi(int i) { return i + ((i >> 4) << PS); }
+__host__ __device__ constexpr int padded_points(int n) { return n + n / 8; }
+__host__ __device__ constexpr int out_shift(int NS) { return NS == 8 ? 1 : 0; }
+// Final-pass outputs (NS >= 64) and caller-written inputs use shift 0.
+__device__ __forceinline__ int pad0(int i) { return padi<0>(i); }
+
 // One pass over registers already holding the inputs of this thread's butterflies:
 //   v[b][r] = data[(t + b T) + r N/R],  T = N/E threads, b < E/R.
 // Applies the pass twiddles (NS = product of earlier radices), the radix-R DFTs,
@@ -120,6 +134,7 @@ __device__ __forceinline__ void pass_from_regs(float2 (*v)[R], float2 *s, int t,
                                                const float2 *__restrict__ tw) {
     constexpr int T = N / E;
     constexpr int NB = E / R;
+    constexpr int PS = out_shift(NS);
 #pragma unroll
     for (int b = 0; b < NB; ++b) {
         const int j = t + b * T;
@@ -131,21 +146,23 @@ __device__ __forceinline__ void pass_from_regs(float2 (*v)[R], float2 *s, int t,
         Dft<R>::run(v[b]);
         const int j0 = (j - k) * R + k;
 #pragma unroll
-        for (int r = 0; r < R; ++r) s[j0 + r * NS] = v[b][r];
+        for (int r = 0; r < R; ++r) s[padi<PS>(j0 + r * NS)] = v[b][r];
     }
 }
 
-// A full pass: gather from `s`, barrier, transform, scatter, barrier.
-template <int N, int E, int R, int NS, typename Sync>
+// A full pass: gather from `s` (laid out by the pass whose NS was NS_PREV; 0 when
+// the caller wrote the input with shift 0), barrier, transform, scatter, barrier.
+template <int N, int E, int R, int NS, int NS_PREV, typename Sync>
 __device__ __forceinline__ void pass(float2 *s, int t, const float2 *__restrict__ tw, Sync sync) {
     constexpr int T = N / E;
     constexpr int NB = E / R;
+    constexpr int PS_IN = out_shift(NS_PREV);
     float2 v[NB][R];
 #pragma unroll
     for (int b = 0; b < NB; ++b) {
         const int j = t + b * T;
 #pragma unroll
-        for (int r = 0; r < R; ++r) v[b][r] = s[j + r * (N / R)];
+        for (int r = 0; r < R; ++r) v[b][r] = s[padi<PS_IN>(j + r * (N / R))];
     }
     sync();
     pass_from_regs<N, E, R, NS>(v, s, t, tw);
