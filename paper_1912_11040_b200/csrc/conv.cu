@@ -97,20 +97,35 @@ __device__ __forceinline__ void mac_pair(float2 &acc_a, float2 &acc_b, float2 a,
 // its stretch of the bank end to end (x[i mod nlen]).  Outside [0, N): zero.
 __device__ __forceinline__ void load_segment(float2 (*v)[8], const float *__restrict__ x, bool looped,
                                              int nlen, int base, int N, int t) {
+    if (!looped) {
 #pragma unroll
-    for (int r = 0; r < 8; ++r) {
-        const int i0 = base + 2 * (t + CT * r);
-        float2 z = make_float2(0.f, 0.f);
-        if (i0 >= 0) {
-            if (!looped) {
+        for (int r = 0; r < 8; ++r) {
+            const int i0 = base + 2 * (t + CT * r);
+            float2 z = make_float2(0.f, 0.f);
+            if (i0 >= 0) {
                 if (i0 + 1 < N) z = *reinterpret_cast<const float2 *>(x + i0);
                 else if (i0 < N) z.x = x[i0];
-            } else {
-                if (i0 < N) z.x = x[i0 % nlen];
-                if (i0 + 1 < N) z.y = x[(i0 + 1) % nlen];
             }
+            v[0][r] = z;
+        }
+        return;
+    }
+    // Looped source: one division for the first sample, then the position advances
+    // by 2*CT (mod nlen) from one pair to the next.
+    const int first = base + 2 * t;
+    const int step = (2 * CT) % nlen;
+    int m = first >= 0 ? first % nlen : (nlen - (-first) % nlen) % nlen;
+#pragma unroll
+    for (int r = 0; r < 8; ++r) {
+        const int i0 = first + 2 * CT * r;
+        float2 z = make_float2(0.f, 0.f);
+        if (i0 >= 0) {
+            if (i0 < N) z.x = x[m];
+            if (i0 + 1 < N) z.y = x[m + 1 == nlen ? 0 : m + 1];
         }
         v[0][r] = z;
+        m += step;
+        if (m >= nlen) m -= nlen;
     }
 }
 

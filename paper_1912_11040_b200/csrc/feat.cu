@@ -237,10 +237,21 @@ frames_kernel(const float *__restrict__ in_a, const float *__restrict__ in_b, in
     if (MODE == 0) {
         for (int i = tid; i < nf * NBP; i += FEAT_THREADS) orow[i] = ptile[i];
     } else {
-        for (int i = tid; i < nf * M; i += FEAT_THREADS) {
-            const int f = i / M, m = i - f * M;
-            orow[i] = compress(band_energy(ptile + f * NBP, mw, mst, m), floor_v, comp);
+        // Filterbank with the lanes of a warp over the frames of the tile: all lanes
+        // of a band walk the same bins (weights are broadcasts, the odd row stride
+        // of ptile keeps the power reads conflict-free, no lane waits for a wider
+        // band).  Results go through shared memory so the global store is contiguous.
+        float *etile = reinterpret_cast<float *>(fbuf);           // [FT][M], transforms are done
+        constexpr int BPW = 32 / FT;                              // bands per warp step
+        const int lane = tid & 31, warp = tid >> 5;
+        const int f = lane % FT, sub = lane / FT;
+        for (int m0 = warp * BPW; m0 < M; m0 += (FEAT_THREADS / 32) * BPW) {
+            const int m = m0 + sub;
+            if (m < M && f < nf)
+                etile[f * M + m] = compress(band_energy(ptile + f * NBP, mw, mst, m), floor_v, comp);
         }
+        __syncthreads();
+        for (int i = tid; i < nf * M; i += FEAT_THREADS) orow[i] = etile[i];
     }
 }
 

@@ -144,9 +144,11 @@ __device__ __forceinline__ void pass_from_regs(float2 (*v)[R], float2 *s, int t,
             twiddle<R>(v[b], w1);
         }
         Dft<R>::run(v[b]);
-        const int j0 = (j - k) * R + k;
+        // Every r * NS is either a multiple of 16 or (NS = 8) stays inside j0's row
+        // pair, so the padded address is padi(j0) plus a compile-time constant.
+        const int base = padi<PS>((j - k) * R + k);
 #pragma unroll
-        for (int r = 0; r < R; ++r) s[padi<PS>(j0 + r * NS)] = v[b][r];
+        for (int r = 0; r < R; ++r) s[base + padi<PS>(r * NS)] = v[b][r];
     }
 }
 
@@ -160,9 +162,10 @@ __device__ __forceinline__ void pass(float2 *s, int t, const float2 *__restrict_
     float2 v[NB][R];
 #pragma unroll
     for (int b = 0; b < NB; ++b) {
-        const int j = t + b * T;
+        static_assert((N / R) % 16 == 0, "gather stride must keep the row offset constant");
+        const int base = padi<PS_IN>(t + b * T);
 #pragma unroll
-        for (int r = 0; r < R; ++r) v[b][r] = s[padi<PS_IN>(j + r * (N / R))];
+        for (int r = 0; r < R; ++r) v[b][r] = s[base + padi<PS_IN>(r * (N / R))];
     }
     sync();
     pass_from_regs<N, E, R, NS>(v, s, t, tw);
