@@ -17,7 +17,7 @@
 //
 // A real transform of F points is a complex transform of F/2 points on (even, odd)
 // sample pairs followed by the usual split; thread t owns the bin pairs
-// (k, F/2-k), k = t + 512 q.  Spectra are stored as F/2 complex numbers with the two
+// (k, F/2-k), k = t + 256 q.  Spectra are stored as F/2 complex numbers with the two
 // real bins (0 and F/2) packed into slot 0.
 #include "common.cuh"
 #include "fft.cuh"
@@ -27,25 +27,23 @@ namespace {
 using namespace augfft;
 constexpr int N2 = aug::CONV_N2;      // 4096 complex points
 constexpr int BLK = aug::CONV_BLK;
-constexpr int CT = 512;               // threads per CTA
-constexpr int E = N2 / CT;            // 8 points per thread
-constexpr int NQ = N2 / 2 / CT;       // 4 bin pairs per thread
+constexpr int CT = 256;               // threads per CTA
+constexpr int E = N2 / CT;            // 16 points per thread: three radix-16 passes
+constexpr int NQ = N2 / 2 / CT;       // 8 bin pairs per thread
 constexpr int SM_POINTS = padded_points(N2);
 
-__device__ __forceinline__ void fft4096_from_regs(float2 (*v)[8], float2 *s, int t,
+__device__ __forceinline__ void fft4096_from_regs(float2 (*v)[E], float2 *s, int t,
                                                   const float2 *__restrict__ tw) {
-    pass_from_regs<N2, E, 8, 1>(v, s, t, tw);
+    pass_from_regs<N2, E, 16, 1>(v, s, t, tw);
     __syncthreads();
-    pass<N2, E, 8, 8, 1>(s, t, tw, CtaSync());
-    pass<N2, E, 8, 64, 8>(s, t, tw, CtaSync());
-    pass<N2, E, 8, 512, 64>(s, t, tw, CtaSync());
+    pass<N2, E, 16, 16, 1>(s, t, tw, CtaSync());
+    pass<N2, E, 16, 256, 16>(s, t, tw, CtaSync());
 }
 
 __device__ __forceinline__ void fft4096_in_place(float2 *s, int t, const float2 *__restrict__ tw) {
-    pass<N2, E, 8, 1, 0>(s, t, tw, CtaSync());
-    pass<N2, E, 8, 8, 1>(s, t, tw, CtaSync());
-    pass<N2, E, 8, 64, 8>(s, t, tw, CtaSync());
-    pass<N2, E, 8, 512, 64>(s, t, tw, CtaSync());
+    pass<N2, E, 16, 1, 0>(s, t, tw, CtaSync());
+    pass<N2, E, 16, 16, 1>(s, t, tw, CtaSync());
+    pass<N2, E, 16, 256, 16>(s, t, tw, CtaSync());
 }
 
 // Split of the half-size transform Z into the spectrum X of the real signal at the
@@ -92,14 +90,14 @@ __device__ __forceinline__ void mac_pair(float2 &acc_a, float2 &acc_b, float2 a,
     acc_b = cadd(acc_b, cmul(b, hb));
 }
 
-// 2*BLK input samples starting at `base` as 8 (even, odd) pairs per thread in the
+// 2*BLK input samples starting at `base` as 16 (even, odd) pairs per thread in the
 // order the first FFT pass wants them.  Speech reads x[i]; a noise source reads
 // its stretch of the bank end to end (x[i mod nlen]).  Outside [0, N): zero.
-__device__ __forceinline__ void load_segment(float2 (*v)[8], const float *__restrict__ x, bool looped,
+__device__ __forceinline__ void load_segment(float2 (*v)[E], const float *__restrict__ x, bool looped,
                                              int nlen, int base, int N, int t) {
     if (!looped) {
 #pragma unroll
-        for (int r = 0; r < 8; ++r) {
+        for (int r = 0; r < E; ++r) {
             const int i0 = base + 2 * (t + CT * r);
             float2 z = make_float2(0.f, 0.f);
             if (i0 >= 0) {
@@ -116,7 +114,7 @@ __device__ __forceinline__ void load_segment(float2 (*v)[8], const float *__rest
     const int step = (2 * CT) % nlen;
     int m = first >= 0 ? first % nlen : (nlen - (-first) % nlen) % nlen;
 #pragma unroll
-    for (int r = 0; r < 8; ++r) {
+    for (int r = 0; r < E; ++r) {
         const int i0 = first + 2 * CT * r;
         float2 z = make_float2(0.f, 0.f);
         if (i0 >= 0) {
@@ -223,9 +221,9 @@ rir_spectra_kernel(const float *__restrict__ rir, const AugUttParams *__restrict
     const float *h = rir + ((int64_t)utt * S_max + s) * L;
     float2 *out = hspec + (((int64_t)utt * S_max + s) * P + p) * N2;
 
-    float2 v[1][8];
+    float2 v[1][E];
 #pragma unroll
-    for (int r = 0; r < 8; ++r) {
+    for (int r = 0; r < E; ++r) {
         const int n = t + CT * r;                 // complex index; taps 2n, 2n+1 of the partition
         const int i0 = p * BLK + 2 * n;
         float2 z = make_float2(0.f, 0.f);
@@ -247,7 +245,7 @@ rir_spectra_kernel(const float *__restrict__ rir, const AugUttParams *__restrict
 }
 
 // ---------------------------------------------------------------- one partition: fused
-__global__ void __launch_bounds__(CT, 2)
+__global__ void __launch_bounds__(CT, 3)
 convolve_fused_kernel(const float *__restrict__ speech, int64_t stride,
                       const int *__restrict__ lengths, const float *__restrict__ bank,
                       int64_t bank_len, const AugUttParams *__restrict__ table, int S_max, int P,
@@ -277,7 +275,7 @@ convolve_fused_kernel(const float *__restrict__ speech, int64_t stride,
                 continue;
             }
             for (int p = 0; p < P && p <= b; ++p) {
-                float2 v[1][8];
+                float2 v[1][E];
                 load_segment(v, x, s != 0, nlen, (b - p - 1) * BLK, N, t);
                 fft4096_from_regs(v, sm, t, tw);
                 const float2 *H = hspec + (((int64_t)utt * S_max + s) * P + p) * N2;
@@ -303,7 +301,7 @@ convolve_fused_kernel(const float *__restrict__ speech, int64_t stride,
 
 // ---------------------------------------------------------------- several partitions
 // Spectrum of every 2*BLK input segment of every source, stored once.
-__global__ void __launch_bounds__(CT, 2)
+__global__ void __launch_bounds__(CT, 3)
 block_spectra_kernel(const float *__restrict__ speech, int64_t stride,
                      const int *__restrict__ lengths, const float *__restrict__ bank,
                      int64_t bank_len, const AugUttParams *__restrict__ table, int S_max,
@@ -321,7 +319,7 @@ block_spectra_kernel(const float *__restrict__ speech, int64_t stride,
         if (t == 0 && b == 0 && atomicCAS(&status[0], -1, utt) == -1) status[1] = aug::R_NOISE;
         return;
     }
-    float2 v[1][8];
+    float2 v[1][E];
     load_segment(v, x, s != 0, nlen, (b - 1) * BLK, N, t);
     fft4096_from_regs(v, sm, t, tw);
     float2 *out = xspec + (((int64_t)utt * S_max + s) * nblk_cap + b) * N2;
@@ -335,7 +333,7 @@ block_spectra_kernel(const float *__restrict__ speech, int64_t stride,
     }
 }
 
-__global__ void __launch_bounds__(CT, 2)
+__global__ void __launch_bounds__(CT, 3)
 spectral_convolve_kernel(const int *__restrict__ lengths, const float *__restrict__ bank,
                          int64_t bank_len, const AugUttParams *__restrict__ table, int S_max, int P,
                          const float2 *__restrict__ hspec, const float2 *__restrict__ xspec,
