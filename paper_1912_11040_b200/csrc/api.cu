@@ -190,11 +190,14 @@ int aug_create(AugCtx **out, const AugConfig *cfg, void *cuda_stream) {
         ctx->st_feats = reinterpret_cast<float *>(base + l.off_st_feats);
         ctx->st_counts = reinterpret_cast<int *>(base + l.off_st_counts);
     }
-    // twiddles exp(-2 pi i m / TW_N), evaluated in double
+    // twiddles, evaluated in double: block [M/2, M) = exp(-2 pi i k / M), k < M/2
     std::vector<float2> tw(augfft::TW_N);
-    for (int m = 0; m < augfft::TW_N; ++m) {
-        const double a = -2.0 * 3.14159265358979323846 * m / augfft::TW_N;
-        tw[m] = make_float2((float)cos(a), (float)sin(a));
+    tw[0] = make_float2(1.f, 0.f);
+    for (int M = 2; M <= augfft::TW_N; M *= 2) {
+        for (int k = 0; k < M / 2; ++k) {
+            const double a = -2.0 * 3.14159265358979323846 * k / M;
+            tw[augfft::tw_index(M, k)] = make_float2((float)cos(a), (float)sin(a));
+        }
     }
     const int st0[2] = {-1, 0};
     bool ok = cudaMemcpyAsync(ctx->tw, tw.data(), sizeof(float2) * augfft::TW_N,

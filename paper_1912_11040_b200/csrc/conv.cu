@@ -63,7 +63,7 @@ __device__ __forceinline__ void real_split(float2 zk, float2 zm, float2 w, float
 __device__ __forceinline__ void spectrum_pair(const float2 *sm, const float2 *__restrict__ tw, int k,
                                               float2 &a, float2 &b) {
     const float2 zk = sm[pad0(k)], zm = sm[pad0((N2 - k) & (N2 - 1))];
-    const float2 w = __ldg(&tw[k * (TW_N / aug::CONV_F)]);
+    const float2 w = __ldg(&tw[tw_index(aug::CONV_F, k)]);
     float2 xk, xm;
     real_split(zk, zm, w, xk, xm);
     if (k == 0) {
@@ -175,7 +175,7 @@ __device__ __forceinline__ void finish_block(const float2 (*acc)[2], float2 *sm,
             sm[pad0(0)] = make_float2(yk.x - yk.y, yk.x + yk.y);
             sm[pad0(N2 / 2)] = make_float2(-2.f * ym.y, 2.f * ym.x);
         } else {
-            const float2 w = __ldg(&tw[k * (TW_N / aug::CONV_F)]);
+            const float2 w = __ldg(&tw[tw_index(aug::CONV_F, k)]);
             // Z[k] = (Yk + conj Ym) + i conj(W)(Yk - conj Ym)
             const float2 a = make_float2(yk.x + ym.x, yk.y - ym.y);
             const float2 d = make_float2(yk.x - ym.x, yk.y + ym.y);

@@ -10,7 +10,11 @@
 
 namespace augfft {
 
-constexpr int TW_N = 16384;  // the twiddle table holds exp(-2 pi i m / TW_N), m < TW_N
+// Twiddle table, TW_N entries: for every power of two M <= TW_N the block
+// [M/2, M) holds exp(-2 pi i k / M), k < M/2, so that the factors one pass or one
+// real-FFT split needs are contiguous in k (coalesced loads).
+constexpr int TW_N = 16384;
+__host__ __device__ constexpr int tw_index(int M, int k) { return M / 2 + k; }
 
 __device__ __forceinline__ float2 cmul(float2 a, float2 b) {
     return make_float2(fmaf(a.x, b.x, -a.y * b.y), fmaf(a.x, b.y, a.y * b.x));
@@ -140,7 +144,7 @@ __device__ __forceinline__ void pass_from_regs(float2 (*v)[R], float2 *s, int t,
         const int j = t + b * T;
         const int k = j & (NS - 1);
         if (NS > 1) {
-            float2 w1 = __ldg(&tw[k * (TW_N / (NS * R))]);
+            float2 w1 = __ldg(&tw[tw_index(NS * R, k)]);
             twiddle<R>(v[b], w1);
         }
         Dft<R>::run(v[b]);
