@@ -5,7 +5,9 @@
 // warp; the 2*W_h+1 taps of each image are then spread over the lanes in fp32:
 // with tau = n0 + phi, sin(pi (n - tau)) = -(-1)^(n-n0) sin(pi phi), so a tap costs
 // one division and a few FMAs, and the Hann factor comes from the angle-sum
-// identity with per-lane constants.
+// identity with per-lane constants.  The lattice points with |kx|+|ky|+|kz| <= order
+// are enumerated compactly (a prefix over kx, then closed forms inside the diamond
+// of (ky, kz)), so every lane of a warp carries a real image.
 #include "common.cuh"
 
 namespace {
@@ -25,7 +27,8 @@ rir_image_kernel(const AugUttParams *__restrict__ table, int S_max, int L, int h
     extern __shared__ __align__(16) unsigned char smem_raw[];
     double *dsq = reinterpret_cast<double *>(smem_raw);   // [3][AX]
     double *gain = dsq + 3 * AX;                          // [3][AX]
-    float *h = reinterpret_cast<float *>(gain + 3 * AX);  // [L]
+    int *xpre = reinterpret_cast<int *>(gain + 3 * AX);   // [AX + 1] images before slab kx
+    float *h = reinterpret_cast<float *>(xpre + AX + 3);  // [L]
 
     const int utt = blockIdx.y, s = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -56,7 +59,17 @@ rir_image_kernel(const AugUttParams *__restrict__ table, int S_max, int L, int h
         gain[a * AX + k + order] = ipow((double)row.beta[2 * a], abs(m - p)) *
                                    ipow((double)row.beta[2 * a + 1], abs(m));
     }
+    if (tid == 0) {
+        int run = 0;
+        for (int ix = 0; ix < side; ++ix) {
+            const int r = order - abs(ix - order);
+            xpre[ix] = run;
+            run += 2 * r * r + 2 * r + 1;      // points of the diamond |ky|+|kz| <= r
+        }
+        xpre[side] = run;
+    }
     __syncthreads();
+    const int total = xpre[side];
 
     // per-lane tap constants: this lane owns taps j = lane + 32 i - half_w
     float cj[3], sj[3], sg[3];
@@ -68,27 +81,42 @@ rir_image_kernel(const AugUttParams *__restrict__ table, int S_max, int L, int h
         sg[i] = (j & 1) ? -1.f : 1.f;
     }
     const float fhw = (float)half_w;
-    const int cube = side * side * side;
     constexpr int NW = RIR_THREADS / 32;
 
-    for (int base = warp * 32; base < cube; base += NW * 32) {
+    for (int base = warp * 32; base < total; base += NW * 32) {
         const int idx = base + lane;
-        bool valid = idx < cube;
+        bool valid = idx < total;
         int n0 = 0;
         float phi = 0.f, A = 0.f, As = 0.f, cph = 0.f, sph = 0.f;
         if (valid) {
-            const int ix = idx / (side * side), rem = idx - ix * side * side;
-            const int iy = rem / side, iz = rem - iy * side;
-            valid = abs(ix - order) + abs(iy - order) + abs(iz - order) <= order;
-            if (valid) {
+            // slab kx: the last ix with xpre[ix] <= idx
+            int lo = 0, hi = side;
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (xpre[mid] <= idx) lo = mid; else hi = mid;
+            }
+            const int ix = lo;
+            const int r = order - abs(ix - order);
+            int q = idx - xpre[ix];                   // position inside the diamond of radius r
+            // rows ky = -r..0 hold 1, 3, .., 2r+1 points (q < (r+1)^2, row u has u^2 before it);
+            // rows ky = 1..r mirror rows r-1..0, counted from the end.
+            const bool upper = q >= (r + 1) * (r + 1);
+            if (upper) q = 2 * r * r + 2 * r - q;
+            int u = (int)sqrtf((float)q);
+            if (u * u > q) --u;
+            if ((u + 1) * (u + 1) <= q) ++u;
+            const int ky = upper ? r - u : u - r;
+            const int kz = q - u * u - u;
+            const int iy = ky + order, iz = kz + order;
+            {
                 const double d = sqrt(dsq[ix] + dsq[AX + iy] + dsq[2 * AX + iz]);
                 const double g = gain[ix] * gain[AX + iy] * gain[2 * AX + iz];
                 const double tau = d * fs / c;
-                const double r = rint(tau);
+                const double rt = rint(tau);
                 A = (float)(g / d);
-                valid = (A != 0.f) && (r - half_w < (double)L);
-                n0 = (int)r;
-                phi = (float)(tau - r);
+                valid = (A != 0.f) && (rt - half_w < (double)L);
+                n0 = (int)rt;
+                phi = (float)(tau - rt);
                 As = -A * sinpif(phi) * 0.318309886183790671538f;
                 cph = 0.5f * cospif(phi / fhw);
                 sph = 0.5f * sinpif(phi / fhw);
@@ -112,7 +140,7 @@ rir_image_kernel(const AugUttParams *__restrict__ table, int S_max, int L, int h
                 const float x = (float)j - phib;
                 if (jj <= 2 * half_w && n >= 0 && n < L && fabsf(x) <= fhw) {
                     const float hann = 0.5f + cj[i] * cb + sj[i] * sb;
-                    const float sc = (fabsf(x) < 1e-7f) ? Ab : sg[i] * Asb / x;
+                    const float sc = (fabsf(x) < 1e-7f) ? Ab : __fdividef(sg[i] * Asb, x);
                     atomicAdd(&h[n], sc * hann);
                 }
             }
@@ -126,12 +154,12 @@ rir_image_kernel(const AugUttParams *__restrict__ table, int S_max, int L, int h
 
 int launch_rir(AugCtx *ctx, const AugUttParams *table, int B, float *rir) {
     const AugConfig &c = ctx->cfg;
-    const size_t smem = sizeof(double) * 6 * AX + sizeof(float) * (size_t)c.rir_taps;
+    const size_t smem = sizeof(double) * 6 * AX + sizeof(int) * (AX + 3) + sizeof(float) * (size_t)c.rir_taps;
     static bool attr_set = false;
     if (!attr_set) {
         AUG_CUDA_OK(cudaFuncSetAttribute(rir_image_kernel,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)(sizeof(double) * 6 * AX + sizeof(float) * aug::MAX_TAPS)));
+                                         (int)(sizeof(double) * 6 * AX + sizeof(int) * (AX + 3) + sizeof(float) * aug::MAX_TAPS)));
         attr_set = true;
     }
     dim3 grid(c.max_sources, B);
