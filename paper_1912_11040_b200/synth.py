@@ -193,7 +193,8 @@ def sample_table(rng, lengths, bank_len, *, room_lo, room_hi, t60, order,
 # --------------------------------------------------------------------------
 
 _COMMON = dict(fs=FS, win=400, hop=160, n_fft=512, n_mel=40, f_lo=0.0, f_hi=FS / 2.0,
-               frac_half_width=40, sound_speed=343.0, log_floor=1e-10, pad_value=0.0,
+               frac_half_width=40, sound_speed=343.0, log_floor=float(np.finfo(np.float32).eps),
+               pad_value=0.0,
                max_sources=S_MAX)
 
 _RECIPES = {

@@ -329,5 +329,5 @@ def test_delta_rir_path_returns_the_input_features():
     assert np.max(np.abs(out["wave"][:lag])) < 1e-15
     assert out["frames"] == 1 + (8000 - 400) // 160
     ref = oracle.logmel(oracle.stft_power(np.concatenate([np.zeros(lag), x[:-lag]]) / d,
-                                          400, 160, 512), 1.0, 512, 40)
+                                          400, 160, 512), 1.0, 512, 40, floor=cfg["log_floor"])
     np.testing.assert_allclose(out["feats"], ref, atol=1e-9)
