@@ -221,10 +221,14 @@ int aug_pipeline(AugCtx *ctx, const float *speech_dev, int64_t speech_stride,
                  int64_t bank_len, const AugUttParams *table_dev, int B, float *feats_dev,
                  int T_max, int *frame_counts_dev, float *wave_out_dev_or_null);
 
-/* Same call for callers that hold HOST buffers: copies speech, lengths, noise
- * bank and table to device staging owned by the context, runs the path, copies
- * feats and frame counts back and synchronises.  Host buffers should be pinned
- * for full copy bandwidth. */
+/* Same call for callers that hold HOST buffers (the context must have been created
+ * with host_staging).  Inputs are copied to device staging owned by the context,
+ * the path runs, feats (padded, [B][T_max][n_mel]) and frame counts are copied
+ * back, and the call returns after synchronising, so the host buffers are free
+ * again.  Internally the batch is cut into up to 8 chunks of utterances that are
+ * copied in, computed and copied out concurrently on three streams; speech rows
+ * are copied only up to their length when that saves more than the extra copy
+ * calls cost.  Host buffers should be pinned for full copy bandwidth. */
 int aug_pipeline_host(AugCtx *ctx, const float *speech_host, int64_t speech_stride,
                       const int *lengths_host, const float *noise_bank_host, int64_t bank_len,
                       const AugUttParams *table_host, int B, float *feats_host, int T_max,
@@ -246,6 +250,9 @@ int aug_stage_times(AugCtx *ctx, float *ms_host, int *n_calls_host);
 
 /* Kernels this context has launched since aug_create. */
 int64_t aug_launch_count(const AugCtx *ctx);
+
+/* Bytes the last aug_pipeline_host call copied host-to-device and device-to-host. */
+int aug_last_host_bytes(const AugCtx *ctx, int64_t *h2d_host, int64_t *d2h_host);
 
 /* Runs a register-resident FMA loop on every SM of the current device and writes
  * the best of three fp32 rates (TFLOP/s, 2 flop per FMA) to *tflops_host.

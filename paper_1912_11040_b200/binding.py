@@ -22,7 +22,7 @@ EXPORTS = ["aug_strerror", "aug_frame_count", "aug_workspace_bytes", "aug_valida
            "aug_create", "aug_destroy", "aug_last_status", "aug_rir_image_method",
            "aug_reverb_mix", "feat_stft_power", "feat_vtlp_logmel", "aug_pipeline",
            "aug_pipeline_host", "aug_enable_stage_timing", "aug_stage_times", "aug_launch_count",
-           "aug_measure_fp32_peak", "feat_vtlp_logmel_noalloc"]
+           "aug_measure_fp32_peak", "feat_vtlp_logmel_noalloc", "aug_last_host_bytes"]
 NOALLOC_MAX_BATCH = 256
 N_STAGES = 6
 STAGE_NAMES = ["rir_image", "rir_spectra", "mel_tables", "convolve", "mix", "features"]
@@ -93,6 +93,8 @@ def lib() -> ctypes.CDLL:
         L.aug_stage_times.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i32)]
         L.aug_launch_count.restype = i64
         L.aug_launch_count.argtypes = [vp]
+        L.aug_last_host_bytes.restype = i32
+        L.aug_last_host_bytes.argtypes = [vp, ctypes.POINTER(i64), ctypes.POINTER(i64)]
         L.aug_measure_fp32_peak.restype = i32
         L.aug_measure_fp32_peak.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
         _lib = L
@@ -234,6 +236,13 @@ class AugContext:
 
     def aug_launch_count(self) -> int:
         return int(lib().aug_launch_count(self._h))
+
+    def aug_last_host_bytes(self):
+        """(host-to-device, device-to-host) bytes of the last aug_pipeline_host call."""
+        a, b = ctypes.c_int64(0), ctypes.c_int64(0)
+        _check(lib().aug_last_host_bytes(self._h, ctypes.byref(a), ctypes.byref(b)),
+               "aug_last_host_bytes")
+        return int(a.value), int(b.value)
 
     def aug_rir_image_method(self, table_dev, B, rir_dev, check=True):
         return self._ret(lib().aug_rir_image_method(self._h, _ptr(table_dev), int(B),

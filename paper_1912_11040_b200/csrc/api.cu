@@ -190,6 +190,19 @@ int aug_create(AugCtx **out, const AugConfig *cfg, void *cuda_stream) {
         ctx->st_feats = reinterpret_cast<float *>(base + l.off_st_feats);
         ctx->st_counts = reinterpret_cast<int *>(base + l.off_st_counts);
     }
+    if (cfg->host_staging) {
+        bool ok_s = cudaStreamCreateWithFlags(&ctx->s_h2d, cudaStreamNonBlocking) == cudaSuccess &&
+                    cudaStreamCreateWithFlags(&ctx->s_d2h, cudaStreamNonBlocking) == cudaSuccess &&
+                    cudaEventCreateWithFlags(&ctx->ev_start, cudaEventDisableTiming) == cudaSuccess;
+        for (int i = 0; i < aug::HOST_CHUNKS && ok_s; ++i)
+            ok_s = cudaEventCreateWithFlags(&ctx->ev_in[i], cudaEventDisableTiming) == cudaSuccess &&
+                   cudaEventCreateWithFlags(&ctx->ev_out[i], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok_s) {
+            cudaFree(ctx->ws_base);
+            delete ctx;
+            return AUG_ECUDA;
+        }
+    }
     // twiddles, evaluated in double: block [M/2, M) = exp(-2 pi i k / M), k < M/2
     std::vector<float2> tw(augfft::TW_N);
     tw[0] = make_float2(1.f, 0.f);
@@ -221,6 +234,17 @@ int aug_destroy(AugCtx *ctx) {
     if (ctx->ev) {
         for (int i = 0; i < aug::EV_RING * (AUG_N_STAGES + 1); ++i) cudaEventDestroy(ctx->ev[i]);
         free(ctx->ev);
+    }
+    if (ctx->s_h2d) {
+        cudaStreamSynchronize(ctx->s_h2d);
+        cudaStreamSynchronize(ctx->s_d2h);
+        for (int i = 0; i < aug::HOST_CHUNKS; ++i) {
+            cudaEventDestroy(ctx->ev_in[i]);
+            cudaEventDestroy(ctx->ev_out[i]);
+        }
+        cudaEventDestroy(ctx->ev_start);
+        cudaStreamDestroy(ctx->s_h2d);
+        cudaStreamDestroy(ctx->s_d2h);
     }
     if (cudaFree(ctx->ws_base) != cudaSuccess) rc = AUG_ECUDA;
     delete ctx;
@@ -349,27 +373,78 @@ int aug_pipeline_host(AugCtx *ctx, const float *speech_host, int64_t speech_stri
     if (speech_stride > ctx->ws_stride || bank_len > ctx->cfg.max_bank_samples || T_max > ctx->t_cap)
         return AUG_ECAP;
     if (bank_len > 0 && !noise_bank_host) return AUG_EINVAL;
-    cudaStream_t st = ctx->stream;
-    AUG_CUDA_OK(cudaMemcpyAsync(ctx->st_speech, speech_host, sizeof(float) * (size_t)B * speech_stride,
-                                cudaMemcpyHostToDevice, st));
+    for (int b = 0; b < B; ++b)
+        if (lengths_host[b] < 0 || lengths_host[b] > speech_stride) return AUG_EINVAL;
+
+    // Software pipeline over chunks of utterances: chunk c+1 is copied in while chunk
+    // c is computed and chunk c-1 is copied out, on three streams tied by events.
+    // Rows are copied only up to their length when the bytes saved outweigh the
+    // cost of one copy call per row.
+    cudaStream_t sc = ctx->stream, si = ctx->s_h2d, so = ctx->s_d2h;
+    int64_t total = 0;
+    for (int b = 0; b < B; ++b) total += lengths_host[b];
+    const double saved_s = (double)((int64_t)B * speech_stride - total) * sizeof(float) / 40e9;
+    const bool ragged = saved_s > (double)B * 4e-6;
+    const int n_chunk = B >= 2 * aug::HOST_CHUNKS ? aug::HOST_CHUNKS : 1;
+
+    AUG_CUDA_OK(cudaEventRecord(ctx->ev_start, sc));          // earlier work on the context's stream
+    AUG_CUDA_OK(cudaStreamWaitEvent(si, ctx->ev_start, 0));
+    AUG_CUDA_OK(cudaMemcpyAsync(ctx->st_table, table_host, sizeof(AugUttParams) * (size_t)B,
+                                cudaMemcpyHostToDevice, si));
+    AUG_CUDA_OK(cudaMemcpyAsync(ctx->st_lengths, lengths_host, sizeof(int) * (size_t)B,
+                                cudaMemcpyHostToDevice, si));
     if (bank_len > 0)
         AUG_CUDA_OK(cudaMemcpyAsync(ctx->st_bank, noise_bank_host, sizeof(float) * (size_t)bank_len,
-                                    cudaMemcpyHostToDevice, st));
-    AUG_CUDA_OK(cudaMemcpyAsync(ctx->st_table, table_host, sizeof(AugUttParams) * (size_t)B,
-                                cudaMemcpyHostToDevice, st));
-    AUG_CUDA_OK(cudaMemcpyAsync(ctx->st_lengths, lengths_host, sizeof(int) * (size_t)B,
-                                cudaMemcpyHostToDevice, st));
-    rc = aug_pipeline(ctx, ctx->st_speech, speech_stride, ctx->st_lengths, lengths_host,
-                      bank_len > 0 ? ctx->st_bank : nullptr, bank_len, ctx->st_table, B,
-                      ctx->st_feats, T_max, ctx->st_counts, nullptr);
+                                    cudaMemcpyHostToDevice, si));
+    const int M = ctx->cfg.n_mel;
+    ctx->last_h2d = (int64_t)sizeof(AugUttParams) * B + (int64_t)sizeof(int) * B +
+                    (int64_t)sizeof(float) * bank_len +
+                    (int64_t)sizeof(float) * (ragged ? total : (int64_t)B * speech_stride);
+    ctx->last_d2h = (int64_t)sizeof(float) * B * T_max * M + (int64_t)sizeof(int) * B;
+    int b0 = 0;
+    int64_t done = 0;
+    for (int c = 0; c < n_chunk; ++c) {
+        // chunk boundaries at equal shares of the samples
+        int b1 = b0;
+        const int64_t goal = total * (c + 1) / n_chunk;
+        while (b1 < B && (done < goal || b1 == b0)) done += lengths_host[b1++];
+        if (c == n_chunk - 1) b1 = B;
+        if (b1 == b0) continue;
+        const int nb = b1 - b0;
+        if (ragged) {
+            for (int b = b0; b < b1; ++b)
+                if (lengths_host[b] > 0)
+                    AUG_CUDA_OK(cudaMemcpyAsync(ctx->st_speech + (int64_t)b * speech_stride,
+                                                speech_host + (int64_t)b * speech_stride,
+                                                sizeof(float) * (size_t)lengths_host[b],
+                                                cudaMemcpyHostToDevice, si));
+        } else {
+            AUG_CUDA_OK(cudaMemcpyAsync(ctx->st_speech + (int64_t)b0 * speech_stride,
+                                        speech_host + (int64_t)b0 * speech_stride,
+                                        sizeof(float) * (size_t)nb * speech_stride,
+                                        cudaMemcpyHostToDevice, si));
+        }
+        AUG_CUDA_OK(cudaEventRecord(ctx->ev_in[c], si));
+        AUG_CUDA_OK(cudaStreamWaitEvent(sc, ctx->ev_in[c], 0));
+        float *f_dev = ctx->st_feats + (int64_t)b0 * T_max * M;
+        rc = aug_pipeline(ctx, ctx->st_speech + (int64_t)b0 * speech_stride, speech_stride,
+                          ctx->st_lengths + b0, lengths_host + b0,
+                          bank_len > 0 ? ctx->st_bank : nullptr, bank_len, ctx->st_table + b0, nb,
+                          f_dev, T_max, ctx->st_counts + b0, nullptr);
+        if (rc != AUG_OK) break;
+        AUG_CUDA_OK(cudaEventRecord(ctx->ev_out[c], sc));
+        AUG_CUDA_OK(cudaStreamWaitEvent(so, ctx->ev_out[c], 0));
+        AUG_CUDA_OK(cudaMemcpyAsync(feats_host + (int64_t)b0 * T_max * M, f_dev,
+                                    sizeof(float) * (size_t)nb * T_max * M, cudaMemcpyDeviceToHost, so));
+        AUG_CUDA_OK(cudaMemcpyAsync(frame_counts_host + b0, ctx->st_counts + b0, sizeof(int) * (size_t)nb,
+                                    cudaMemcpyDeviceToHost, so));
+        b0 = b1;
+    }
+    // drain all three streams whatever happened above
+    const bool ok = cudaStreamSynchronize(si) == cudaSuccess && cudaStreamSynchronize(sc) == cudaSuccess &&
+                    cudaStreamSynchronize(so) == cudaSuccess;
     if (rc != AUG_OK) return rc;
-    AUG_CUDA_OK(cudaMemcpyAsync(feats_host, ctx->st_feats,
-                                sizeof(float) * (size_t)B * T_max * ctx->cfg.n_mel,
-                                cudaMemcpyDeviceToHost, st));
-    AUG_CUDA_OK(cudaMemcpyAsync(frame_counts_host, ctx->st_counts, sizeof(int) * (size_t)B,
-                                cudaMemcpyDeviceToHost, st));
-    AUG_CUDA_OK(cudaStreamSynchronize(st));
-    return AUG_OK;
+    return ok ? AUG_OK : AUG_ECUDA;
 }
 
 int aug_enable_stage_timing(AugCtx *ctx, int on) {
@@ -412,5 +487,12 @@ int aug_stage_times(AugCtx *ctx, float *ms_host, int *n_calls_host) {
 }
 
 int64_t aug_launch_count(const AugCtx *ctx) { return ctx ? ctx->launches : 0; }
+
+int aug_last_host_bytes(const AugCtx *ctx, int64_t *h2d_host, int64_t *d2h_host) {
+    if (!ctx) return AUG_EINVAL;
+    if (h2d_host) *h2d_host = ctx->last_h2d;
+    if (d2h_host) *d2h_host = ctx->last_d2h;
+    return AUG_OK;
+}
 
 }  // extern "C"

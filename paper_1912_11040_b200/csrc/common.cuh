@@ -16,6 +16,7 @@ constexpr int MAX_HALF_W = 47;
 constexpr int MAX_MEL = 128;
 
 constexpr int EV_RING = 256;
+constexpr int HOST_CHUNKS = 8;           // pipeline depth of aug_pipeline_host
 
 enum Reason { R_NONE = 0, R_NSRC = 1, R_ORDER = 2, R_NOISE = 3, R_WAIT = 4 };
 
@@ -63,6 +64,9 @@ struct AugCtx {
     int *st_lengths;
     float *st_feats;       // [max_batch][t_cap][n_mel]
     int *st_counts;
+    int64_t last_h2d, last_d2h;                // bytes the last aug_pipeline_host call copied
+    cudaStream_t s_h2d, s_d2h;                 // copy streams of the host-buffer entry point
+    cudaEvent_t ev_in[aug::HOST_CHUNKS], ev_out[aug::HOST_CHUNKS], ev_start;
 };
 
 #define AUG_CUDA_OK(expr)                         \

@@ -105,6 +105,7 @@ __device__ __forceinline__ void tile_power(const float *chunk, int nf, int win, 
         const int n = tg + GROUP * r;
         wv[r] = n < win ? 0.5f - 0.5f * cospif(2.f * (float)n / (float)win) : 0.f;
     }
+    const GroupSync gsync{grp + 1, GROUP};
     const int npair = (nf + 1) / 2;
     const int iters = (npair + NGROUP - 1) / NGROUP;
     for (int it = 0; it < iters; ++it) {
@@ -122,16 +123,17 @@ __device__ __forceinline__ void tile_power(const float *chunk, int nf, int win, 
             }
             v[0][r] = make_float2(a, b);
         }
+        // each 64-thread group runs its transforms on its own hardware barrier
         if constexpr (K == 512) {
             pass_from_regs<K, E, 8, 1>(v, s, tg, tw);
-            __syncthreads();
-            pass<K, E, 8, 8, 1>(s, tg, tw, CtaSync());
-            pass<K, E, 8, 64, 8>(s, tg, tw, CtaSync());
+            gsync();
+            pass<K, E, 8, 8, 1>(s, tg, tw, gsync);
+            pass<K, E, 8, 64, 8>(s, tg, tw, gsync);
         } else {
             pass_from_regs<K, E, E, 1>(v, s, tg, tw);
-            __syncthreads();
-            pass<K, E, 8, 16, 1>(s, tg, tw, CtaSync());
-            pass<K, E, 8, 128, 16>(s, tg, tw, CtaSync());
+            gsync();
+            pass<K, E, 8, 16, 1>(s, tg, tw, gsync);
+            pass<K, E, 8, 128, 16>(s, tg, tw, gsync);
         }
         if (have0) {
             float *p0 = ptile + f0 * NBP, *p1 = p0 + NBP;
@@ -143,8 +145,9 @@ __device__ __forceinline__ void tile_power(const float *chunk, int nf, int win, 
                 if (have1) p1[k] = 0.25f * (br * br + bi * bi);
             }
         }
-        __syncthreads();
+        gsync();   // the group's buffer is rewritten by its next pair
     }
+    __syncthreads();   // all power spectra of the tile are in place
 }
 
 template <int K>

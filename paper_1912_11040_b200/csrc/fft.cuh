@@ -179,5 +179,12 @@ __device__ __forceinline__ void pass(float2 *s, int t, const float2 *__restrict_
 struct CtaSync {
     __device__ __forceinline__ void operator()() const { __syncthreads(); }
 };
+// Barrier over `count` threads (whole warps) that share hardware barrier `id` (1..15).
+struct GroupSync {
+    int id, count;
+    __device__ __forceinline__ void operator()() const {
+        asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+    }
+};
 
 }  // namespace augfft
