@@ -43,20 +43,44 @@ def workload_label(i):
 
 # ------------------------------------------------------------------ algorithmic work
 def conv_work(w):
-    """Nominal flops and compulsory bytes of the convolution kernel for one batch:
-    per source one forward real FFT per 4096-sample block (2.5 F log2 F, F = 8192),
+    """Nominal flops and compulsory bytes of the convolution step for one batch, per kernel.
+    Per source one forward real FFT per 4096-sample block (2.5 F log2 F, F = 8192),
     8 flops per bin and partition for the spectral multiply-accumulate, two inverse
-    FFTs per block; bytes = inputs read once + y_s and v written once + the
-    partition spectra read once."""
+    FFTs per block.  With one partition a single fused kernel does all of it
+    (bytes: inputs read once, y_s and v written once, partition spectra read once);
+    with more, block_spectra_kernel does the forward FFTs (inputs in, block spectra
+    out) and spectral_convolve_kernel the rest (block and partition spectra in,
+    y_s and v out)."""
     F, blk = 8192, 4096
     P = -(-int(w.cfg["rir_taps"]) // blk)
     fft = 2.5 * F * 13
-    flops = bytes_ = 0.0
+    spec = (F // 2) * 8.0
+    fwd_f = fwd_b = fin_f = fin_b = 0.0
     for b in range(w.B):
         n, S = int(w.lengths[b]), int(w.table["n_src"][b])
         nblk = -(-n // blk)
-        flops += nblk * (S * (fft + 8.0 * (F // 2) * P) + (2 if S > 1 else 1) * fft)
-        bytes_ += 4.0 * n * S + 4.0 * n * 2 + S * P * (F // 2) * 8.0
+        fwd_f += nblk * S * fft
+        fin_f += nblk * (S * 8.0 * (F // 2) * P + (2 if S > 1 else 1) * fft)
+        if P == 1:
+            fin_b += 4.0 * n * S + 4.0 * n * 2 + S * P * spec
+        else:
+            fwd_b += 4.0 * n * S + nblk * S * spec
+            fin_b += nblk * S * spec + S * P * spec + 4.0 * n * 2
+    if P == 1:
+        return {"convolve": (fwd_f + fin_f, fin_b)}
+    return {"block_spectra": (fwd_f, fwd_b), "convolve": (fin_f, fin_b)}
+
+
+def rir_work(w):
+    """Image-method kernel: ~10 flops per tap, 2 W_h + 1 taps per image; bytes = responses out."""
+    taps = 2 * int(w.cfg["frac_half_width"]) + 1
+    flops = bytes_ = 0.0
+    for b in range(w.B):
+        n = int(w.table["order"][b])
+        images = (2 * n + 1) * (2 * n * n + 2 * n + 3) // 3
+        S = int(w.table["n_src"][b])
+        flops += 10.0 * taps * images * S
+        bytes_ += 4.0 * int(w.cfg["rir_taps"]) * S
     return flops, bytes_
 
 
@@ -291,7 +315,11 @@ def run_ours(args):
     hbm_peak, hbm_src = (peaks["hbm_gbs"], "measured") if "hbm_gbs" in peaks else (6650.0, "fallback")
     fp32_measured = binding.aug_measure_fp32_peak()
     fp32_nominal = SM_COUNT * FP32_LANES * 2 * (clocks["sm_max_mhz"] or 1965) * 1e6 / 1e12
-    kernels = {"convolve": (3, conv_work(w)), "features": (5, feat_work(w))}
+    idx_of = {n: i for i, n in enumerate(binding.STAGE_NAMES)}
+    work = dict(conv_work(w))
+    work["features"] = feat_work(w)
+    work["rir_image"] = rir_work(w)
+    kernels = {name: (idx_of[name], fb) for name, fb in work.items()}
     dom = max(kernels, key=lambda k: stage_ms[kernels[k][0]])
     per_kernel = {}
     for name, (idx, (flops, byts)) in kernels.items():

@@ -237,8 +237,9 @@ int aug_pipeline_host(AugCtx *ctx, const float *speech_host, int64_t speech_stri
 /* -------------------------------------------------------------- measurement utilities
  * (instrumentation of this library; the paper has no counterpart) */
 
-#define AUG_N_STAGES 6 /* 0 impulse responses, 1 partition spectra, 2 filterbank tables,
-                          3 convolution, 4 waveform mix (only when requested), 5 features */
+#define AUG_N_STAGES 7 /* 0 impulse responses, 1 partition spectra, 2 filterbank tables,
+                          3 block spectra of the audio (multi-partition responses only),
+                          4 convolution, 5 waveform mix (only when requested), 6 features */
 
 /* on != 0: aug_pipeline records CUDA events between its kernels (up to 256 calls
  * are kept); on == 0: stop.  Either way the record is cleared. */

@@ -24,8 +24,9 @@ EXPORTS = ["aug_strerror", "aug_frame_count", "aug_workspace_bytes", "aug_valida
            "aug_pipeline_host", "aug_enable_stage_timing", "aug_stage_times", "aug_launch_count",
            "aug_measure_fp32_peak", "feat_vtlp_logmel_noalloc", "aug_last_host_bytes"]
 NOALLOC_MAX_BATCH = 256
-N_STAGES = 6
-STAGE_NAMES = ["rir_image", "rir_spectra", "mel_tables", "convolve", "mix", "features"]
+N_STAGES = 7
+STAGE_NAMES = ["rir_image", "rir_spectra", "mel_tables", "block_spectra", "convolve", "mix",
+               "features"]
 
 
 class AugConfig(ctypes.Structure):

@@ -232,9 +232,10 @@ int aug_destroy(AugCtx *ctx) {
     int rc = AUG_OK;
     if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) rc = AUG_ECUDA;
     if (ctx->ev) {
-        for (int i = 0; i < aug::EV_RING * (AUG_N_STAGES + 1); ++i) cudaEventDestroy(ctx->ev[i]);
+        for (int i = 0; i < aug::EV_RING * 2 * AUG_N_STAGES; ++i) cudaEventDestroy(ctx->ev[i]);
         free(ctx->ev);
     }
+
     if (ctx->s_h2d) {
         cudaStreamSynchronize(ctx->s_h2d);
         cudaStreamSynchronize(ctx->s_d2h);
@@ -269,7 +270,7 @@ int aug_rir_image_method(AugCtx *ctx, const AugUttParams *table_dev, int B, floa
     if (rc != AUG_OK) return rc;
     if (B == 0) return AUG_OK;
     if (!table_dev || !rir_dev || !aligned16(rir_dev)) return AUG_EINVAL;
-    return launch_rir(ctx, table_dev, B, rir_dev);
+    return launch_rir(ctx, table_dev, B, rir_dev, ctx->stream);
 }
 
 int aug_reverb_mix(AugCtx *ctx, const float *speech_dev, int64_t speech_stride,
@@ -284,9 +285,11 @@ int aug_reverb_mix(AugCtx *ctx, const float *speech_dev, int64_t speech_stride,
     if (speech_stride <= 0 || (speech_stride & 3) || bank_len < 0) return AUG_EINVAL;
     const int max_len = (int)(speech_stride < ctx->cfg.max_samples ? speech_stride : ctx->cfg.max_samples);
     if (speech_stride > ctx->ws_stride) return AUG_ECAP;
-    if ((rc = launch_rir_spectra(ctx, rir_dev, table_dev, B)) != AUG_OK) return rc;
-    if ((rc = launch_convolve(ctx, speech_dev, speech_stride, lengths_dev, noise_bank_dev, bank_len,
-                              table_dev, B, max_len)) != AUG_OK) return rc;
+    if ((rc = launch_rir_spectra(ctx, rir_dev, table_dev, B, ctx->stream)) != AUG_OK) return rc;
+    if ((rc = launch_convolve_prepare(ctx, speech_dev, speech_stride, lengths_dev, noise_bank_dev,
+                                      bank_len, table_dev, B, max_len)) != AUG_OK) return rc;
+    if ((rc = launch_convolve_finish(ctx, speech_dev, speech_stride, lengths_dev, noise_bank_dev,
+                                     bank_len, table_dev, B, max_len)) != AUG_OK) return rc;
     return launch_mix(ctx, lengths_dev, table_dev, B, max_len, wave_out_dev, speech_stride);
 }
 
@@ -307,7 +310,7 @@ int feat_vtlp_logmel(AugCtx *ctx, const float *power_dev, const int *frame_count
     if (rc != AUG_OK) return rc;
     if (B == 0) return AUG_OK;
     if (!power_dev || !frame_counts_dev || !table_dev || !feats_dev || T_max <= 0) return AUG_EINVAL;
-    if ((rc = launch_mel_tables(ctx, table_dev, B)) != AUG_OK) return rc;
+    if ((rc = launch_mel_tables(ctx, table_dev, B, ctx->stream)) != AUG_OK) return rc;
     return launch_logmel(ctx, power_dev, frame_counts_dev, B, T_max, feats_dev);
 }
 
@@ -335,27 +338,46 @@ int aug_pipeline(AugCtx *ctx, const float *speech_dev, int64_t speech_stride,
         if (aug_frame_count(mx, ctx->cfg.win, ctx->cfg.hop) > T_max) return AUG_ECAP;
         max_len = mx;
     }
+    // Stage timing: a start and a stop event per stage, on the stream the stage runs on.
     cudaEvent_t *ev = nullptr;
     if (ctx->timing && ctx->ev && ctx->ev_n < aug::EV_RING)
-        ev = ctx->ev + (size_t)ctx->ev_n * (AUG_N_STAGES + 1);
-    auto mark = [&](int i) { if (ev) cudaEventRecord(ev[i], ctx->stream); };
-    mark(0);
-    if ((rc = launch_rir(ctx, table_dev, B, ctx->rir)) != AUG_OK) return rc;
-    mark(1);
-    if ((rc = launch_rir_spectra(ctx, ctx->rir, table_dev, B)) != AUG_OK) return rc;
-    mark(2);
-    if ((rc = launch_mel_tables(ctx, table_dev, B)) != AUG_OK) return rc;
-    mark(3);
-    if ((rc = launch_convolve(ctx, speech_dev, speech_stride, lengths_dev, noise_bank_dev, bank_len,
-                              table_dev, B, max_len)) != AUG_OK) return rc;
-    mark(4);
+        ev = ctx->ev + (size_t)ctx->ev_n * (2 * AUG_N_STAGES);
+    auto t0 = [&](int stage, cudaStream_t st) { if (ev) cudaEventRecord(ev[2 * stage], st); };
+    auto t1 = [&](int stage, cudaStream_t st) { if (ev) cudaEventRecord(ev[2 * stage + 1], st); };
+    // One stream: running the impulse-response chain beside the block spectra on a
+    // second stream was measured and gained nothing (both saturate the SMs' issue
+    // and shared-memory pipes), so the stages simply follow one another.
+    cudaStream_t sm = ctx->stream, ss = ctx->stream;
+    t0(0, ss);
+    rc = launch_rir(ctx, table_dev, B, ctx->rir, ss);
+    t1(0, ss);
+    t0(1, ss);
+    if (rc == AUG_OK) rc = launch_rir_spectra(ctx, ctx->rir, table_dev, B, ss);
+    t1(1, ss);
+    t0(2, ss);
+    if (rc == AUG_OK) rc = launch_mel_tables(ctx, table_dev, B, ss);
+    t1(2, ss);
+
+    t0(3, sm);
+    if (rc == AUG_OK)
+        rc = launch_convolve_prepare(ctx, speech_dev, speech_stride, lengths_dev, noise_bank_dev,
+                                     bank_len, table_dev, B, max_len);
+    t1(3, sm);
+    if (rc != AUG_OK) return rc;
+    t0(4, sm);
+    rc = launch_convolve_finish(ctx, speech_dev, speech_stride, lengths_dev, noise_bank_dev, bank_len,
+                                table_dev, B, max_len);
+    t1(4, sm);
+    if (rc != AUG_OK) return rc;
+    t0(5, sm);
     if (wave_out &&
         (rc = launch_mix(ctx, lengths_dev, table_dev, B, max_len, wave_out, speech_stride)) != AUG_OK)
         return rc;
-    mark(5);
+    t1(5, sm);
+    t0(6, sm);
     rc = launch_fused_features(ctx, lengths_dev, table_dev, B, feats_dev, T_max, frame_counts_dev,
                                nullptr, 0);
-    mark(6);
+    t1(6, sm);
     if (ev && rc == AUG_OK) ctx->ev_n++;
     return rc;
 }
@@ -451,7 +473,7 @@ int aug_enable_stage_timing(AugCtx *ctx, int on) {
     if (!ctx) return AUG_EINVAL;
     AUG_CUDA_OK(cudaStreamSynchronize(ctx->stream));
     if (on && !ctx->ev) {
-        const int n = aug::EV_RING * (AUG_N_STAGES + 1);
+        const int n = aug::EV_RING * 2 * AUG_N_STAGES;
         ctx->ev = static_cast<cudaEvent_t *>(calloc(n, sizeof(cudaEvent_t)));
         if (!ctx->ev) return AUG_ENOMEM;
         for (int i = 0; i < n; ++i) {
@@ -473,10 +495,10 @@ int aug_stage_times(AugCtx *ctx, float *ms_host, int *n_calls_host) {
     AUG_CUDA_OK(cudaStreamSynchronize(ctx->stream));
     double acc[AUG_N_STAGES] = {0};
     for (int c = 0; c < ctx->ev_n; ++c) {
-        cudaEvent_t *ev = ctx->ev + (size_t)c * (AUG_N_STAGES + 1);
+        cudaEvent_t *ev = ctx->ev + (size_t)c * (2 * AUG_N_STAGES);
         for (int i = 0; i < AUG_N_STAGES; ++i) {
             float ms = 0.f;
-            AUG_CUDA_OK(cudaEventElapsedTime(&ms, ev[i], ev[i + 1]));
+            AUG_CUDA_OK(cudaEventElapsedTime(&ms, ev[2 * i], ev[2 * i + 1]));
             acc[i] += ms;
         }
     }

@@ -55,7 +55,7 @@ struct AugCtx {
     // instrumentation
     int64_t launches;      // kernels launched so far
     int timing;            // record events between the stages of aug_pipeline
-    cudaEvent_t *ev;       // [EV_RING][AUG_N_STAGES + 1]
+    cudaEvent_t *ev;       // [EV_RING][2 * AUG_N_STAGES]: start and stop of every stage
     int ev_n;              // calls recorded
     // staging for the host-buffer entry point (NULL unless cfg.host_staging)
     float *st_speech;      // [max_batch][ws_stride]
@@ -75,15 +75,23 @@ struct AugCtx {
         if (e__ != cudaSuccess) return AUG_ECUDA; \
     } while (0)
 
-// Launchers (defined next to their kernels).  All enqueue on ctx->stream.
-int launch_rir(AugCtx *ctx, const AugUttParams *table, int B, float *rir);
-int launch_rir_spectra(AugCtx *ctx, const float *rir, const AugUttParams *table, int B);
-int launch_convolve(AugCtx *ctx, const float *speech, int64_t stride, const int *lengths,
-                    const float *bank, int64_t bank_len, const AugUttParams *table, int B,
-                    int max_len);
+// Launchers (defined next to their kernels).  They enqueue on ctx->stream unless a
+// stream is passed.
+int launch_rir(AugCtx *ctx, const AugUttParams *table, int B, float *rir, cudaStream_t st);
+int launch_rir_spectra(AugCtx *ctx, const float *rir, const AugUttParams *table, int B,
+                       cudaStream_t st);
+// Convolution in two parts: `prepare` needs only the input audio (block spectra when
+// the response has several partitions, else nothing), `finish` also needs the
+// partition spectra of the impulse responses.
+int launch_convolve_prepare(AugCtx *ctx, const float *speech, int64_t stride, const int *lengths,
+                            const float *bank, int64_t bank_len, const AugUttParams *table, int B,
+                            int max_len);
+int launch_convolve_finish(AugCtx *ctx, const float *speech, int64_t stride, const int *lengths,
+                           const float *bank, int64_t bank_len, const AugUttParams *table, int B,
+                           int max_len);
 int launch_mix(AugCtx *ctx, const int *lengths, const AugUttParams *table, int B, int max_len,
                float *wave_out, int64_t out_stride);
-int launch_mel_tables(AugCtx *ctx, const AugUttParams *table, int B);
+int launch_mel_tables(AugCtx *ctx, const AugUttParams *table, int B, cudaStream_t st);
 int launch_stft_power(AugCtx *ctx, const float *wave, int64_t stride, const int *lengths, int B,
                       float *power, int T_max, int *counts);
 int launch_logmel(AugCtx *ctx, const float *power, const int *counts, int B, int T_max,

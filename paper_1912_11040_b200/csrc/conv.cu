@@ -31,6 +31,9 @@ constexpr int CT = 256;               // threads per CTA
 constexpr int E = N2 / CT;            // 16 points per thread: three radix-16 passes
 constexpr int NQ = N2 / 2 / CT;       // 8 bin pairs per thread
 constexpr int SM_POINTS = padded_points(N2);
+#ifndef CONV_MINB
+#define CONV_MINB 3                  // CTAs per SM the register budget is set for
+#endif
 
 __device__ __forceinline__ void fft4096_from_regs(float2 (*v)[E], float2 *s, int t,
                                                   const float2 *__restrict__ tw) {
@@ -245,7 +248,7 @@ rir_spectra_kernel(const float *__restrict__ rir, const AugUttParams *__restrict
 }
 
 // ---------------------------------------------------------------- one partition: fused
-__global__ void __launch_bounds__(CT, 3)
+__global__ void __launch_bounds__(CT, CONV_MINB)
 convolve_fused_kernel(const float *__restrict__ speech, int64_t stride,
                       const int *__restrict__ lengths, const float *__restrict__ bank,
                       int64_t bank_len, const AugUttParams *__restrict__ table, int S_max, int P,
@@ -301,7 +304,7 @@ convolve_fused_kernel(const float *__restrict__ speech, int64_t stride,
 
 // ---------------------------------------------------------------- several partitions
 // Spectrum of every 2*BLK input segment of every source, stored once.
-__global__ void __launch_bounds__(CT, 3)
+__global__ void __launch_bounds__(CT, CONV_MINB)
 block_spectra_kernel(const float *__restrict__ speech, int64_t stride,
                      const int *__restrict__ lengths, const float *__restrict__ bank,
                      int64_t bank_len, const AugUttParams *__restrict__ table, int S_max,
@@ -333,7 +336,7 @@ block_spectra_kernel(const float *__restrict__ speech, int64_t stride,
     }
 }
 
-__global__ void __launch_bounds__(CT, 3)
+__global__ void __launch_bounds__(CT, CONV_MINB)
 spectral_convolve_kernel(const int *__restrict__ lengths, const float *__restrict__ bank,
                          int64_t bank_len, const AugUttParams *__restrict__ table, int S_max, int P,
                          const float2 *__restrict__ hspec, const float2 *__restrict__ xspec,
@@ -416,42 +419,52 @@ constexpr size_t FFT_SMEM = sizeof(float2) * SM_POINTS;
 
 }  // namespace
 
-int launch_rir_spectra(AugCtx *ctx, const float *rir, const AugUttParams *table, int B) {
+int launch_rir_spectra(AugCtx *ctx, const float *rir, const AugUttParams *table, int B,
+                       cudaStream_t st) {
     const AugConfig &c = ctx->cfg;
     dim3 grid(ctx->n_part, c.max_sources, B);
-    rir_spectra_kernel<<<grid, CT, FFT_SMEM, ctx->stream>>>(rir, table, c.max_sources, c.rir_taps,
+    rir_spectra_kernel<<<grid, CT, FFT_SMEM, st>>>(rir, table, c.max_sources, c.rir_taps,
                                                             ctx->n_part, ctx->tw, ctx->hspec);
     AUG_CUDA_OK(cudaGetLastError());
     ctx->launches++;
     return AUG_OK;
 }
 
-int launch_convolve(AugCtx *ctx, const float *speech, int64_t stride, const int *lengths,
-                    const float *bank, int64_t bank_len, const AugUttParams *table, int B,
-                    int max_len) {
+static bool stored_route(const AugCtx *ctx) { return ctx->n_part > 1 && ctx->xspec != nullptr; }
+
+int launch_convolve_prepare(AugCtx *ctx, const float *speech, int64_t stride, const int *lengths,
+                            const float *bank, int64_t bank_len, const AugUttParams *table, int B,
+                            int max_len) {
     const AugConfig &c = ctx->cfg;
     if (max_len <= 0) return AUG_OK;
     AUG_CUDA_OK(cudaMemsetAsync(ctx->energy, 0, sizeof(double) * 2 * (size_t)B, ctx->stream));
+    if (!stored_route(ctx)) return AUG_OK;
     const int nblk = (max_len + BLK - 1) / BLK;
-    if (ctx->n_part == 1 || ctx->xspec == nullptr) {
-        dim3 grid(nblk, B);
-        convolve_fused_kernel<<<grid, CT, FFT_SMEM, ctx->stream>>>(
-            speech, stride, lengths, bank, bank_len, table, c.max_sources, ctx->n_part, ctx->hspec,
-            ctx->tw, ctx->ys, ctx->vv, ctx->ws_stride, ctx->energy, ctx->status, max_len);
-        AUG_CUDA_OK(cudaGetLastError());
-        ctx->launches++;
-        return AUG_OK;
-    }
     dim3 grid_x(nblk, c.max_sources, B);
     block_spectra_kernel<<<grid_x, CT, FFT_SMEM, ctx->stream>>>(
         speech, stride, lengths, bank, bank_len, table, c.max_sources, ctx->tw, ctx->xspec,
         ctx->nblk_cap, ctx->status, max_len);
     AUG_CUDA_OK(cudaGetLastError());
     ctx->launches++;
+    return AUG_OK;
+}
+
+int launch_convolve_finish(AugCtx *ctx, const float *speech, int64_t stride, const int *lengths,
+                           const float *bank, int64_t bank_len, const AugUttParams *table, int B,
+                           int max_len) {
+    const AugConfig &c = ctx->cfg;
+    if (max_len <= 0) return AUG_OK;
+    const int nblk = (max_len + BLK - 1) / BLK;
     dim3 grid(nblk, B);
-    spectral_convolve_kernel<<<grid, CT, FFT_SMEM, ctx->stream>>>(
-        lengths, bank, bank_len, table, c.max_sources, ctx->n_part, ctx->hspec, ctx->xspec,
-        ctx->nblk_cap, ctx->tw, ctx->ys, ctx->vv, ctx->ws_stride, ctx->energy, max_len);
+    if (!stored_route(ctx)) {
+        convolve_fused_kernel<<<grid, CT, FFT_SMEM, ctx->stream>>>(
+            speech, stride, lengths, bank, bank_len, table, c.max_sources, ctx->n_part, ctx->hspec,
+            ctx->tw, ctx->ys, ctx->vv, ctx->ws_stride, ctx->energy, ctx->status, max_len);
+    } else {
+        spectral_convolve_kernel<<<grid, CT, FFT_SMEM, ctx->stream>>>(
+            lengths, bank, bank_len, table, c.max_sources, ctx->n_part, ctx->hspec, ctx->xspec,
+            ctx->nblk_cap, ctx->tw, ctx->ys, ctx->vv, ctx->ws_stride, ctx->energy, max_len);
+    }
     AUG_CUDA_OK(cudaGetLastError());
     ctx->launches++;
     return AUG_OK;

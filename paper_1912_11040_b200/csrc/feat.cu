@@ -309,9 +309,9 @@ int launch_frames(AugCtx *ctx, const float *a, const float *b, int64_t stride, c
 
 }  // namespace
 
-int launch_mel_tables(AugCtx *ctx, const AugUttParams *table, int B) {
+int launch_mel_tables(AugCtx *ctx, const AugUttParams *table, int B, cudaStream_t st) {
     const AugConfig &c = ctx->cfg;
-    mel_tables_kernel<<<B, 256, 0, ctx->stream>>>(table, c.n_fft, c.n_mel, (double)c.fs,
+    mel_tables_kernel<<<B, 256, 0, st>>>(table, c.n_fft, c.n_mel, (double)c.fs,
                                                   (double)c.f_lo, (double)c.f_hi, ctx->melw,
                                                   ctx->melstart);
     AUG_CUDA_OK(cudaGetLastError());

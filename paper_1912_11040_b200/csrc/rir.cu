@@ -152,7 +152,7 @@ rir_image_kernel(const AugUttParams *__restrict__ table, int S_max, int L, int h
 
 }  // namespace
 
-int launch_rir(AugCtx *ctx, const AugUttParams *table, int B, float *rir) {
+int launch_rir(AugCtx *ctx, const AugUttParams *table, int B, float *rir, cudaStream_t st) {
     const AugConfig &c = ctx->cfg;
     const size_t smem = sizeof(double) * 6 * AX + sizeof(int) * (AX + 3) + sizeof(float) * (size_t)c.rir_taps;
     static bool attr_set = false;
@@ -163,7 +163,7 @@ int launch_rir(AugCtx *ctx, const AugUttParams *table, int B, float *rir) {
         attr_set = true;
     }
     dim3 grid(c.max_sources, B);
-    rir_image_kernel<<<grid, RIR_THREADS, smem, ctx->stream>>>(
+    rir_image_kernel<<<grid, RIR_THREADS, smem, st>>>(
         table, c.max_sources, c.rir_taps, c.frac_half_width, (double)c.fs, (double)c.sound_speed,
         c.max_order, rir, ctx->status);
     AUG_CUDA_OK(cudaGetLastError());
