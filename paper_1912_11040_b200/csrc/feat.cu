@@ -150,15 +150,21 @@ __device__ __forceinline__ void tile_power(const float *chunk, int nf, int win, 
     __syncthreads();   // all power spectra of the tile are in place
 }
 
+#ifndef FEAT_FT_512
+#define FEAT_FT_512 32      // frames per CTA tile, 512-point transform
+#endif
+#ifndef FEAT_FT_1024
+#define FEAT_FT_1024 16     // frames per CTA tile, 1024-point transform
+#endif
 template <int K>
 struct Plan;
 template <>
 struct Plan<512> {
-    static constexpr int E = 8, FT = 32;
+    static constexpr int E = 8, FT = FEAT_FT_512;
 };
 template <>
 struct Plan<1024> {
-    static constexpr int E = 16, FT = 16;
+    static constexpr int E = 16, FT = FEAT_FT_1024;
 };
 
 __device__ __forceinline__ float snr_gain_f(const double *energy, int utt, int n_src, float snr_db) {
