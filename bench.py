@@ -32,6 +32,21 @@ METRIC = "audio-seconds augmented+featurised per second"
 UNIT = "audio-s/s"
 SM_COUNT, FP32_LANES = 148, 128
 
+# DRAM bytes per audio-second of workload 2 (dram__bytes_read.sum + dram__bytes_write.sum of one
+# ncu --set full capture on 96 utterances; traffic grows in proportion to the audio processed).
+# Valid only for the kernel sources the capture was taken from: the hash guards that.
+NCU_TRAFFIC = {"workload": 2, "sources_sha": "f7eb0b1a28015847",
+               "bytes_per_audio_s": {"convolve": 466.58e6 / 1039.18, "block_spectra": 403.27e6 / 1039.18,
+                                     "features": 148.79e6 / 1039.18, "rir_image": 0.04e6 / 1039.18}}
+
+
+def kernel_sources_sha():
+    import hashlib
+    h = hashlib.sha256()
+    for f in ("conv.cu", "fft.cuh", "feat.cu", "rir.cu"):
+        h.update(open(os.path.join(ROOT, "paper_1912_11040_b200", "csrc", f), "rb").read())
+    return h.hexdigest()[:16]
+
 
 def workload_label(i):
     return {1: "config1: 8 x 2 s, order 6, 4096 taps, 1 white noise, 40 mel",
@@ -342,6 +357,11 @@ def run_ours(args):
         roofline = {"kernel": dom, "bound": "hbm", "achieved": d["gbs"], "peak": hbm_peak,
                     "unit": "GB/s", "frac": d["frac_hbm"], "traffic": None,
                     "peak_source": f"{hbm_src} copy bandwidth"}
+    if (args.workload == NCU_TRAFFIC["workload"] and dom in NCU_TRAFFIC["bytes_per_audio_s"]
+            and kernel_sources_sha() == NCU_TRAFFIC["sources_sha"]):
+        roofline["traffic"] = NCU_TRAFFIC["bytes_per_audio_s"][dom] * w.audio_seconds
+        roofline["traffic_note"] = ("bytes per launch, ncu capture on 96 utterances scaled by audio-seconds; "
+                                    "algorithmic bytes of this kernel: %.3e" % kernels[dom][1][1])
     roofline["per_kernel"] = per_kernel
     roofline["stage_ms"] = dict(zip(binding.STAGE_NAMES, stage_ms))
     roofline["stage_calls_averaged"] = n_rec
