@@ -222,6 +222,20 @@ def run_reference(args):
     return 0
 
 
+def combine_ranks(audio_seconds, ms_device, s_e2e, world, device):
+    """Whole-job figures from per-rank ones: every rank is an independent replica, so
+    the audio processed adds up and the job takes as long as its slowest rank."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([audio_seconds, ms_device, s_e2e], dtype=torch.float64, device=device)
+    if world > 1:
+        a = t.clone()
+        dist.all_reduce(a[0:1], op=dist.ReduceOp.SUM)
+        dist.all_reduce(a[1:3], op=dist.ReduceOp.MAX)
+        t = a
+    return tuple(float(v) for v in t.cpu())
+
+
 # ------------------------------------------------------------------ GPU arm
 def run_ours(args):
     import torch
@@ -305,14 +319,7 @@ def run_ours(args):
     barrier()
     h2d, d2h = ctx.aug_last_host_bytes()     # what the library really copied (ragged rows)
 
-    # ---- reduce over ranks: max time, summed audio
-    audio = torch.tensor([w.audio_seconds, ms_total, dt_e2e], dtype=torch.float64, device="cuda")
-    if world > 1:
-        a = audio.clone()
-        dist.all_reduce(a[0:1], op=dist.ReduceOp.SUM)
-        dist.all_reduce(a[1:3], op=dist.ReduceOp.MAX)
-        audio = a
-    audio_total, ms_total, dt_e2e = (float(v) for v in audio.cpu())
+    audio_total, ms_total, dt_e2e = combine_ranks(w.audio_seconds, ms_total, dt_e2e, world, "cuda")
     value = audio_total * args.steps / (ms_total * 1e-3)
     e2e_value = audio_total * e2e_steps / dt_e2e
 

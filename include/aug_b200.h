@@ -113,6 +113,32 @@ int64_t aug_workspace_bytes(const AugConfig *cfg_host);
 int aug_validate_params(const AugConfig *cfg_host, const AugUttParams *table_host, int B,
                         int64_t bank_len, int *bad_row_host);
 
+/* Ranges the per-utterance parameters are drawn from (uniformly, independently):
+ * the "millions of room dimensions, wide distribution of reverberation time and
+ * SNR" of Section 1 and the random warp factor of Section 2.3. */
+typedef struct {
+    float room_lo[3], room_hi[3]; /* shoebox side lengths, metres */
+    float t60_lo, t60_hi;         /* reverberation time, seconds; turned into one wall reflection
+                                     coefficient by Eyring's formula */
+    int32_t order;                /* reflection order written to every row */
+    int32_t n_noise_lo, n_noise_hi; /* noise sources per utterance, 0..AUG_S_MAX-1 */
+    float snr_lo, snr_hi;         /* dB */
+    float alpha_lo, alpha_hi;     /* VTLP warp factor (Table 2 of the paper tries 0.8..1.2) */
+    float wall_margin;            /* microphone and sources keep this distance from the walls */
+    float min_src_mic_dist;       /* sources are redrawn while closer than this to the microphone */
+    int32_t min_noise_len;        /* shortest stretch of the noise bank a source may loop */
+    int64_t bank_len;             /* samples in the noise bank the offsets refer to */
+} AugDist;
+
+/* Draw B rows on the host from `seed` (counter-based SplitMix64: row b depends only
+ * on seed and b).  Each noise source gets a stretch of the bank of length between
+ * half the utterance and the whole utterance (clamped to [min_noise_len, bank_len])
+ * at a uniform offset, weight 1.  Rows always pass aug_validate_params for a
+ * configuration with max_order >= order and max_sources > n_noise_hi.
+ * Returns AUG_EINVAL for null pointers or inconsistent ranges. */
+int aug_sample_params(uint64_t seed, const AugDist *dist_host, int B, const int *lengths_host,
+                      AugUttParams *table_host);
+
 /* -------------------------------------------------------------- context */
 
 /* Create a context for cfg on the current CUDA device; cuda_stream is a

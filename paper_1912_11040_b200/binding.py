@@ -22,7 +22,7 @@ EXPORTS = ["aug_strerror", "aug_frame_count", "aug_workspace_bytes", "aug_valida
            "aug_create", "aug_destroy", "aug_last_status", "aug_rir_image_method",
            "aug_reverb_mix", "feat_stft_power", "feat_vtlp_logmel", "aug_pipeline",
            "aug_pipeline_host", "aug_enable_stage_timing", "aug_stage_times", "aug_launch_count",
-           "aug_measure_fp32_peak", "feat_vtlp_logmel_noalloc", "aug_last_host_bytes"]
+           "aug_measure_fp32_peak", "feat_vtlp_logmel_noalloc", "aug_last_host_bytes", "aug_sample_params"]
 NOALLOC_MAX_BATCH = 256
 N_STAGES = 7
 STAGE_NAMES = ["rir_image", "rir_spectra", "mel_tables", "block_spectra", "convolve", "mix",
@@ -39,6 +39,16 @@ class AugConfig(ctypes.Structure):
                 ("compression", ctypes.c_int32), ("max_batch", ctypes.c_int32),
                 ("max_samples", ctypes.c_int32), ("host_staging", ctypes.c_int32),
                 ("max_bank_samples", ctypes.c_int64)]
+
+
+class AugDist(ctypes.Structure):
+    _fields_ = [("room_lo", ctypes.c_float * 3), ("room_hi", ctypes.c_float * 3),
+                ("t60_lo", ctypes.c_float), ("t60_hi", ctypes.c_float), ("order", ctypes.c_int32),
+                ("n_noise_lo", ctypes.c_int32), ("n_noise_hi", ctypes.c_int32),
+                ("snr_lo", ctypes.c_float), ("snr_hi", ctypes.c_float),
+                ("alpha_lo", ctypes.c_float), ("alpha_hi", ctypes.c_float),
+                ("wall_margin", ctypes.c_float), ("min_src_mic_dist", ctypes.c_float),
+                ("min_noise_len", ctypes.c_int32), ("bank_len", ctypes.c_int64)]
 
 
 class AugError(RuntimeError):
@@ -94,6 +104,8 @@ def lib() -> ctypes.CDLL:
         L.aug_stage_times.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i32)]
         L.aug_launch_count.restype = i64
         L.aug_launch_count.argtypes = [vp]
+        L.aug_sample_params.restype = i32
+        L.aug_sample_params.argtypes = [ctypes.c_uint64, ctypes.POINTER(AugDist), i32, vp, vp]
         L.aug_last_host_bytes.restype = i32
         L.aug_last_host_bytes.argtypes = [vp, ctypes.POINTER(i64), ctypes.POINTER(i64)]
         L.aug_measure_fp32_peak.restype = i32
@@ -134,6 +146,17 @@ def aug_validate_params(config: AugConfig, table: np.ndarray, bank_len: int):
     rc = lib().aug_validate_params(ctypes.byref(config), table.ctypes.data, int(table.shape[0]),
                                    int(bank_len), ctypes.byref(bad))
     return int(rc), int(bad.value)
+
+
+def aug_sample_params(seed: int, dist: AugDist, lengths: np.ndarray, check: bool = True):
+    """Draw one table row per utterance on the host; returns (status, table)."""
+    lengths = np.ascontiguousarray(lengths, dtype=np.int32)
+    table = np.zeros(lengths.shape[0], dtype=UTT_DTYPE)
+    rc = int(lib().aug_sample_params(ctypes.c_uint64(int(seed)), ctypes.byref(dist),
+                                     int(lengths.shape[0]), lengths.ctypes.data, table.ctypes.data))
+    if check:
+        _check(rc, "aug_sample_params")
+    return rc, table
 
 
 def aug_measure_fp32_peak(stream: Optional[int] = None) -> float:

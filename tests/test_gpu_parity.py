@@ -176,3 +176,28 @@ def test_errors_and_status_word():
     assert dev.ctx.aug_last_status() == (1, 1)
     assert dev.ctx.aug_last_status() == (-1, 0)
     assert not rir[1].any()
+
+
+def test_pipeline_runs_on_a_table_from_the_library_sampler():
+    """aug_sample_params rows drive the kernels without a rejected row; results are
+    finite and padded.  (Parity inputs never come from the library: those are synth's.)"""
+    w = small(2, batch=16, dur_scale=0.1)
+    d = binding.AugDist()
+    d.room_lo[:] = (3, 3, 2.5)
+    d.room_hi[:] = (10, 10, 5)
+    d.t60_lo, d.t60_hi, d.order = 0.1, 0.9, int(w.cfg["max_order"])
+    d.n_noise_lo, d.n_noise_hi = 0, 3
+    d.snr_lo, d.snr_hi, d.alpha_lo, d.alpha_hi = 0, 30, 0.8, 1.2
+    d.wall_margin, d.min_src_mic_dist, d.min_noise_len, d.bank_len = 0.3, 0.5, 4000, w.bank.size
+    _, w.table = binding.aug_sample_params(123, d, w.lengths)
+    dev = Device(w)
+    assert binding.aug_validate_params(dev.cfg, w.table, w.bank.size) == (0, -1)
+    F, counts, wave = dev.pipeline(want_wave=True)
+    assert dev.ctx.aug_last_status() == (-1, 0)
+    F, counts, wave = F.cpu().numpy(), counts.cpu().numpy(), wave.cpu().numpy()
+    for b in range(w.B):
+        T = binding.aug_frame_count(int(w.lengths[b]), 400, 160)
+        assert counts[b] == T
+        assert np.all(np.isfinite(F[b, :T])) and np.all(F[b, T:] == 0.0)
+        assert np.all(np.isfinite(wave[b, : w.lengths[b]]))
+        assert np.sqrt(np.mean(wave[b, : w.lengths[b]] ** 2)) > 1e-5

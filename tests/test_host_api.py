@@ -82,6 +82,67 @@ def test_validate_params():
     assert binding.aug_validate_params(cfg, w.table, 10)[0] == binding.AUG_EPARAM  # bank too short
 
 
+def _dist(bank_len=200000, **kw):
+    d = binding.AugDist()
+    d.room_lo[:] = (3, 3, 2.5)
+    d.room_hi[:] = (10, 8, 4)
+    d.t60_lo, d.t60_hi, d.order = 0.2, 0.8, 6
+    d.n_noise_lo, d.n_noise_hi = 0, 3
+    d.snr_lo, d.snr_hi, d.alpha_lo, d.alpha_hi = 0, 20, 0.8, 1.2
+    d.wall_margin, d.min_src_mic_dist, d.min_noise_len, d.bank_len = 0.3, 0.5, 4000, bank_len
+    for k, v in kw.items():
+        setattr(d, k, v)
+    return d
+
+
+def test_sample_params_rows_are_valid_deterministic_and_in_range():
+    rng = np.random.default_rng(0)
+    lengths = rng.integers(1000, 160000, 500).astype(np.int32)
+    d = _dist()
+    rc, t = binding.aug_sample_params(7, d, lengths)
+    assert rc == 0
+    w = synth.make_workload(2, batch=1, dur_scale=0.05)
+    cfg = binding.make_config(dict(w.cfg, max_order=6, max_sources=4), 500, 160000)
+    assert binding.aug_validate_params(cfg, t, d.bank_len) == (0, -1)
+    assert np.all((t["room"] >= (3, 3, 2.5)) & (t["room"] <= (10, 8, 4)))
+    assert np.all((t["alpha"] >= 0.8) & (t["alpha"] <= 1.2)) and np.all((t["snr_db"] >= 0) & (t["snr_db"] <= 20))
+    assert set(np.unique(t["n_src"])) == {1, 2, 3, 4} and np.all(t["order"] == 6)
+    # Eyring: the drawn beta corresponds to a T60 inside the requested range
+    vol = t["room"].astype(np.float64).prod(axis=1)
+    r = t["room"].astype(np.float64)
+    surf = 2 * (r[:, 0] * r[:, 1] + r[:, 1] * r[:, 2] + r[:, 0] * r[:, 2])
+    t60 = -0.161 * vol / (surf * np.log(t["beta"][:, 0].astype(np.float64) ** 2))
+    assert np.all((t60 > 0.2 - 1e-4) & (t60 < 0.8 + 1e-4))
+    assert np.all(t["beta"] == t["beta"][:, :1])
+    # geometry: margins and minimum distance
+    assert np.all(t["mic"] >= 0.3 - 1e-6) and np.all(t["mic"] <= t["room"] - 0.3 + 1e-6)
+    for s in range(4):
+        used = t["n_src"] > s
+        dist = np.linalg.norm(t["src_pos"][used, s] - t["mic"][used], axis=1)
+        assert np.all(dist >= 0.5 - 1e-5)
+    # noise stretches: inside the bank, between half and the whole utterance (floored at 4000)
+    for j in range(3):
+        used = t["n_src"] > j + 1
+        ln, n = t["noise_len"][used, j], np.maximum(lengths[used], 4000)
+        assert np.all(ln <= n) and np.all(ln >= np.maximum(n // 2, 4000))
+        assert np.all(t["noise_offset"][used, j] + ln <= d.bank_len)
+    # counter-based: a row depends on (seed, row index) only
+    _, t2 = binding.aug_sample_params(7, d, lengths[:10])
+    assert t2.tobytes() == t[:10].tobytes()
+    _, t3 = binding.aug_sample_params(8, d, lengths[:10])
+    assert t3.tobytes() != t[:10].tobytes()
+    # the draws look uniform: mean alpha near the middle of its range
+    assert abs(float(t["alpha"].mean()) - 1.0) < 0.03
+
+
+def test_sample_params_rejects_bad_ranges():
+    lengths = np.full(4, 16000, dtype=np.int32)
+    assert binding.aug_sample_params(0, _dist(alpha_hi=2.5), lengths, check=False)[0] == binding.AUG_EINVAL
+    assert binding.aug_sample_params(0, _dist(n_noise_hi=4), lengths, check=False)[0] == binding.AUG_EINVAL
+    assert binding.aug_sample_params(0, _dist(t60_lo=0.0), lengths, check=False)[0] == binding.AUG_EINVAL
+    assert binding.aug_sample_params(0, _dist(bank_len=0), lengths, check=False)[0] == binding.AUG_EINVAL
+
+
 def test_compute_calls_refuse_without_a_gpu():
     import torch
     if torch.cuda.is_available():
