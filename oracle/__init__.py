@@ -34,22 +34,25 @@ from . import build as _build
 _lib = None
 
 
+def _bind(lib):
+    dp = ctypes.POINTER(ctypes.c_double)
+    lib.orc_rir_image_method.restype = ctypes.c_int64
+    lib.orc_rir_image_method.argtypes = [dp, dp, dp, dp, ctypes.c_int, ctypes.c_double,
+                                         ctypes.c_double, ctypes.c_int, ctypes.c_int, dp]
+    lib.orc_convolve_causal.restype = None
+    lib.orc_convolve_causal.argtypes = [dp, ctypes.c_int64, dp, ctypes.c_int64, dp]
+    lib.orc_frame_count.restype = ctypes.c_int
+    lib.orc_frame_count.argtypes = [ctypes.c_int64, ctypes.c_int, ctypes.c_int]
+    lib.orc_stft_power.restype = None
+    lib.orc_stft_power.argtypes = [dp, ctypes.c_int64, ctypes.c_int, ctypes.c_int,
+                                   ctypes.c_int, dp]
+    return lib
+
+
 def _load():
     global _lib
     if _lib is None:
-        lib = ctypes.CDLL(_build.build())
-        dp = ctypes.POINTER(ctypes.c_double)
-        lib.orc_rir_image_method.restype = ctypes.c_int64
-        lib.orc_rir_image_method.argtypes = [dp, dp, dp, dp, ctypes.c_int, ctypes.c_double,
-                                             ctypes.c_double, ctypes.c_int, ctypes.c_int, dp]
-        lib.orc_convolve_causal.restype = None
-        lib.orc_convolve_causal.argtypes = [dp, ctypes.c_int64, dp, ctypes.c_int64, dp]
-        lib.orc_frame_count.restype = ctypes.c_int
-        lib.orc_frame_count.argtypes = [ctypes.c_int64, ctypes.c_int, ctypes.c_int]
-        lib.orc_stft_power.restype = None
-        lib.orc_stft_power.argtypes = [dp, ctypes.c_int64, ctypes.c_int, ctypes.c_int,
-                                       ctypes.c_int, dp]
-        _lib = lib
+        _lib = _bind(ctypes.CDLL(_build.build()))
     return _lib
 
 

@@ -108,6 +108,32 @@ def test_fractional_delay_kernel_delays_a_sinusoid():
     assert np.max(np.abs(y[600:] - ref[600:])) < 1e-3 / d
 
 
+def test_delay_kernel_window_shape():
+    # One image, delay exactly n0 + 1/2 (d = 343/32000 * (2 n0 + 1), exact in binary for n0 = 100:
+    # d = 2.15446875 is not, so the half-sample is checked to 1e-9 instead of assumed).
+    n0 = 100
+    d = C / FS * (n0 + 0.5)
+    room, mic = [30.0, 30.0, 30.0], [10.0, 10.0, 10.0]
+    for hw in (40, 41):
+        h = oracle.rir_image_method(room, [0.0] * 6, mic, [10.0 + d, 10.0, 10.0], 0, 512,
+                                    half_width=hw) * d
+        tau = d * FS / C
+        assert abs(tau - (n0 + 0.5)) < 1e-9
+        # support: 2*hw taps for a half-sample delay, nothing beyond |n - tau| <= hw
+        nz = np.nonzero(h)[0]
+        assert nz[0] == n0 - hw + 1 and nz[-1] == n0 + hw
+        # a Hann window closes smoothly: the outermost taps are tiny but not zero
+        for edge in (n0 - hw + 1, n0 + hw):
+            assert 1e-9 < abs(h[edge]) < 1e-5
+        # the two taps next to the delay: sinc(1/2) = 2/pi, window ~ 1
+        assert h[n0] == pytest.approx(2 / np.pi, rel=2e-3) and h[n0 + 1] == pytest.approx(2 / np.pi, rel=2e-3)
+        # symmetric about the delay
+        np.testing.assert_allclose(h[n0 - hw + 1: n0 + 1], h[n0 + 1: n0 + hw + 1][::-1], rtol=1e-9)
+    # half width 41: |n - tau| = 20.5 is half the window, where a Hann window equals 1/2 exactly
+    # and sinc(20.5) = 1/(20.5 pi) in magnitude
+    assert abs(h[n0 + 21]) == pytest.approx(0.5 / (20.5 * np.pi), rel=1e-9)
+
+
 def test_rir_taps_outside_the_buffer_are_dropped():
     room, mic, src = [5.0, 4.0, 3.0], [1.0, 1.2, 1.1], [3.3, 2.9, 1.7]
     beta = [0.8] * 6
