@@ -48,6 +48,11 @@ typedef enum {
 
 typedef enum { AUG_COMPRESS_LOG = 0, AUG_COMPRESS_POW_1_15 = 1 } AugCompression;
 
+/* Which image sources a reflection order N keeps: those reached by at most N
+ * reflections in total (|kx|+|ky|+|kz| <= N, the default), or the whole cube
+ * max(|kx|,|ky|,|kz|) <= N, up to 3N reflections: (2N+1)^3 images, a stress mode. */
+typedef enum { AUG_LATTICE_TOTAL = 0, AUG_LATTICE_CUBE = 1 } AugLattice;
+
 /* Fixed at aug_create.  Plain data, no pointers. */
 typedef struct {
     int32_t fs;              /* sampling rate, Hz */
@@ -68,6 +73,7 @@ typedef struct {
     int32_t max_batch;       /* capacity: utterances per call */
     int32_t max_samples;     /* capacity: samples per utterance */
     int32_t host_staging;    /* non-zero: also allocate device staging for aug_pipeline_host */
+    int32_t image_lattice;   /* AugLattice */
     int64_t max_bank_samples; /* capacity of the staged noise bank (host_staging only) */
 } AugConfig;
 
@@ -160,7 +166,8 @@ int aug_last_status(AugCtx *ctx, int *utt_host, int *reason_host);
  * Room impulse responses by the image-source method (simulator block, Sections
  * 1 and 2.3; computed on the fly per utterance as Section 1 requires).
  *   rir_dev [B][max_sources][rir_taps] fp32, overwritten; sources >= n_src get zeros.
- * For each source the sum runs over the image lattice |kx|+|ky|+|kz| <= order;
+ * For each source the sum runs over the image lattice |kx|+|ky|+|kz| <= order
+ * (or the cube, see AugLattice);
  * an image at distance d adds (prod beta^hits / d) times a Hann-windowed sinc
  * (half width frac_half_width) centred at d*fs/sound_speed samples. */
 int aug_rir_image_method(AugCtx *ctx, const AugUttParams *table_dev, int B, float *rir_dev);
@@ -235,6 +242,28 @@ int feat_vtlp_logmel(AugCtx *ctx, const float *power_dev, const int *frame_count
 int feat_vtlp_logmel_noalloc(const AugConfig *cfg_host, const float *power_dev,
                              const int *frame_counts_dev, const AugUttParams *table_dev, int B,
                              int T_max, float *feats_dev, void *cuda_stream);
+
+/* -------------------------------------------------------------- after the features
+ * Cepstra: orthonormal DCT-II of each feature row (the MFCC baseline of Table 1
+ * when the features are log-mel):  c_i = s_i sum_m x[m] cos(pi i (m + 1/2) / n_mel),
+ * s_0 = sqrt(1/n_mel), s_i = sqrt(2/n_mel), i < n_cep <= n_mel.
+ *   feats_dev [B][T_max][n_mel] -> mfcc_dev [B][T_max][n_cep]; rows t >= frame_counts[b]
+ *   receive pad_value. */
+int feat_mfcc(AugCtx *ctx, const float *feats_dev, const int *frame_counts_dev, int B, int T_max,
+              int n_cep, float *mfcc_dev);
+
+/* Per-utterance mean and (population) variance of each of D features over the
+ * frame_counts[b] valid frames: mean_dev, var_dev [B][D]; both 0 for an utterance
+ * without frames.  Sums are carried in fp64. */
+int feat_mean_var(AugCtx *ctx, const float *feats_dev, const int *frame_counts_dev, int B, int T_max,
+                  int D, float *mean_dev, float *var_dev);
+
+/* Host only.  Padded batches of similar length (Section 2.2): perm_host[B] lists the
+ * utterances by increasing length (stable), so consecutive groups of `batch` entries
+ * pad least; batch_max_host[ceil(B/batch)] (may be NULL) receives each group's
+ * longest length. */
+int aug_bucket_by_length(const int *lengths_host, int B, int batch, int *perm_host,
+                         int *batch_max_host);
 
 /* -------------------------------------------------------------- steps 1-4
  * The whole path for a batch.  Arguments as above; additionally

@@ -37,7 +37,7 @@ _lib = None
 def _bind(lib):
     dp = ctypes.POINTER(ctypes.c_double)
     lib.orc_rir_image_method.restype = ctypes.c_int64
-    lib.orc_rir_image_method.argtypes = [dp, dp, dp, dp, ctypes.c_int, ctypes.c_double,
+    lib.orc_rir_image_method.argtypes = [dp, dp, dp, dp, ctypes.c_int, ctypes.c_int, ctypes.c_double,
                                          ctypes.c_double, ctypes.c_int, ctypes.c_int, dp]
     lib.orc_convolve_causal.restype = None
     lib.orc_convolve_causal.argtypes = [dp, ctypes.c_int64, dp, ctypes.c_int64, dp]
@@ -63,15 +63,17 @@ def _d(a):
 
 # ---------------------------------------------------------------- step 1
 def rir_image_method(room, beta, mic, src, order, taps, fs=16000.0, c=343.0, half_width=40,
-                     return_count=False):
-    """h[taps]: sum over image sources with |kx|+|ky|+|kz| <= order of
+                     return_count=False, lattice="total"):
+    """h[taps]: sum over image sources with |kx|+|ky|+|kz| <= order (lattice "total") or
+    max(|kx|,|ky|,|kz|) <= order (lattice "cube") of
     (prod beta^hits / d) * Hann-windowed sinc centred at d*fs/c."""
     room, pr = _d(room)
     beta, pb = _d(beta)
     mic, pm = _d(mic)
     src, ps = _d(src)
     h = np.zeros(int(taps), dtype=np.float64)
-    n = _load().orc_rir_image_method(pr, pb, pm, ps, int(order), float(fs), float(c),
+    assert lattice in ("total", "cube")
+    n = _load().orc_rir_image_method(pr, pb, pm, ps, int(order), int(lattice == "cube"), float(fs), float(c),
                                      int(half_width), int(taps),
                                      h.ctypes.data_as(ctypes.POINTER(ctypes.c_double)))
     return (h, int(n)) if return_count else h
@@ -177,6 +179,28 @@ def logmel(power, alpha, n_fft, n_mel, fs=16000.0, f_lo=0.0, f_hi=None, floor=1e
     raise ValueError(compression)
 
 
+# ---------------------------------------------------------------- after the features
+def mfcc(feats, n_cep):
+    """Orthonormal DCT-II of every row: c_i = s_i sum_m x[m] cos(pi i (m + 1/2)/M),
+    s_0 = sqrt(1/M), s_i = sqrt(2/M) (the MFCC baseline of Table 1 when x is log-mel)."""
+    feats = np.asarray(feats, dtype=np.float64)
+    M = feats.shape[-1]
+    i = np.arange(int(n_cep))[:, None]
+    m = np.arange(M)[None, :]
+    C = np.cos(np.pi * i * (m + 0.5) / M) * np.sqrt(2.0 / M)
+    C[0] *= np.sqrt(0.5)
+    return feats @ C.T
+
+
+def mean_var(feats):
+    """Mean and population variance of each feature over the frames; zeros without frames."""
+    feats = np.asarray(feats, dtype=np.float64)
+    if feats.shape[0] == 0:
+        return np.zeros(feats.shape[1]), np.zeros(feats.shape[1])
+    mu = feats.sum(axis=0) / feats.shape[0]
+    return mu, ((feats - mu) ** 2).sum(axis=0) / feats.shape[0]
+
+
 # ---------------------------------------------------------------- whole path
 def utterance(speech, bank, row, cfg, compression="log"):
     """One utterance through all four steps.  `row` is one record of the parameter
@@ -186,7 +210,8 @@ def utterance(speech, bank, row, cfg, compression="log"):
     n_src = int(row["n_src"])
     rirs = [rir_image_method(row["room"], row["beta"], row["mic"], row["src_pos"][s],
                              int(row["order"]), int(cfg["rir_taps"]), fs,
-                             float(cfg["sound_speed"]), int(cfg["frac_half_width"]))
+                             float(cfg["sound_speed"]), int(cfg["frac_half_width"]),
+                             lattice=cfg.get("image_lattice", "total"))
             for s in range(n_src)]
     n = len(speech)
     noises = [looped_noise(bank, row["noise_offset"][k], row["noise_len"][k], n)

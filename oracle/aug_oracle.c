@@ -38,7 +38,8 @@ static double sinc_pi(double x) {
  *
  *   room[3]  side lengths in metres
  *   beta[6]  pressure reflection coefficients of the walls x=0, x=Lx, y=0, y=Ly, z=0, z=Lz
- *   order    largest total number of reflections |kx|+|ky|+|kz| kept
+ *   order    largest total number of reflections |kx|+|ky|+|kz| kept (cube == 0), or
+ *            largest per-axis index max(|kx|,|ky|,|kz|) (cube != 0)
  *   half_w   half width W_h (samples) of the Hann-windowed sinc that places a
  *            delay tau between sample points
  *   h[L]     output, overwritten
@@ -50,14 +51,14 @@ static double sinc_pi(double x) {
  * Returns the number of images summed.
  */
 int64_t orc_rir_image_method(const double *room, const double *beta, const double *mic,
-                             const double *src, int order, double fs, double c,
+                             const double *src, int order, int cube, double fs, double c,
                              int half_w, int L, double *h) {
     int64_t n_img = 0;
     memset(h, 0, sizeof(double) * (size_t)L);
     for (int kx = -order; kx <= order; ++kx)
         for (int ky = -order; ky <= order; ++ky)
             for (int kz = -order; kz <= order; ++kz) {
-                if (abs(kx) + abs(ky) + abs(kz) > order) continue;
+                if (!cube && abs(kx) + abs(ky) + abs(kz) > order) continue;
                 int k[3] = {kx, ky, kz};
                 double d2 = 0.0, gain = 1.0;
                 for (int a = 0; a < 3; ++a) {

@@ -17,12 +17,14 @@ LIB_PATH = os.path.join(_HERE, "libaugb200.so")
 
 AUG_OK, AUG_EINVAL, AUG_ECAP, AUG_ECUDA, AUG_EPARAM, AUG_ENOMEM = 0, -1, -2, -3, -4, -5
 COMPRESS_LOG, COMPRESS_POW_1_15 = 0, 1
+LATTICE_TOTAL, LATTICE_CUBE = 0, 1
 
 EXPORTS = ["aug_strerror", "aug_frame_count", "aug_workspace_bytes", "aug_validate_params",
            "aug_create", "aug_destroy", "aug_last_status", "aug_rir_image_method",
            "aug_reverb_mix", "feat_stft_power", "feat_vtlp_logmel", "aug_pipeline",
            "aug_pipeline_host", "aug_enable_stage_timing", "aug_stage_times", "aug_launch_count",
-           "aug_measure_fp32_peak", "feat_vtlp_logmel_noalloc", "aug_last_host_bytes", "aug_sample_params"]
+           "aug_measure_fp32_peak", "feat_vtlp_logmel_noalloc", "aug_last_host_bytes", "aug_sample_params", "feat_mfcc", "feat_mean_var",
+           "aug_bucket_by_length"]
 NOALLOC_MAX_BATCH = 256
 N_STAGES = 7
 STAGE_NAMES = ["rir_image", "rir_spectra", "mel_tables", "block_spectra", "convolve", "mix",
@@ -38,7 +40,7 @@ class AugConfig(ctypes.Structure):
                 ("log_floor", ctypes.c_float), ("pad_value", ctypes.c_float),
                 ("compression", ctypes.c_int32), ("max_batch", ctypes.c_int32),
                 ("max_samples", ctypes.c_int32), ("host_staging", ctypes.c_int32),
-                ("max_bank_samples", ctypes.c_int64)]
+                ("image_lattice", ctypes.c_int32), ("max_bank_samples", ctypes.c_int64)]
 
 
 class AugDist(ctypes.Structure):
@@ -104,6 +106,12 @@ def lib() -> ctypes.CDLL:
         L.aug_stage_times.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i32)]
         L.aug_launch_count.restype = i64
         L.aug_launch_count.argtypes = [vp]
+        L.feat_mfcc.restype = i32
+        L.feat_mfcc.argtypes = [vp, vp, vp, i32, i32, i32, vp]
+        L.feat_mean_var.restype = i32
+        L.feat_mean_var.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp]
+        L.aug_bucket_by_length.restype = i32
+        L.aug_bucket_by_length.argtypes = [vp, i32, i32, vp, vp]
         L.aug_sample_params.restype = i32
         L.aug_sample_params.argtypes = [ctypes.c_uint64, ctypes.POINTER(AugDist), i32, vp, vp]
         L.aug_last_host_bytes.restype = i32
@@ -123,7 +131,8 @@ def aug_frame_count(n_samples: int, win: int, hop: int) -> int:
 
 
 def make_config(cfg: dict, max_batch: int, max_samples: int, *, compression: int = COMPRESS_LOG,
-                host_staging: bool = False, max_bank_samples: int = 0) -> AugConfig:
+                host_staging: bool = False, max_bank_samples: int = 0,
+                image_lattice: int = LATTICE_TOTAL) -> AugConfig:
     return AugConfig(fs=int(cfg["fs"]), win=int(cfg["win"]), hop=int(cfg["hop"]),
                      n_fft=int(cfg["n_fft"]), n_mel=int(cfg["n_mel"]), f_lo=float(cfg["f_lo"]),
                      f_hi=float(cfg["f_hi"]), rir_taps=int(cfg["rir_taps"]),
@@ -132,7 +141,8 @@ def make_config(cfg: dict, max_batch: int, max_samples: int, *, compression: int
                      sound_speed=float(cfg["sound_speed"]), log_floor=float(cfg["log_floor"]),
                      pad_value=float(cfg["pad_value"]), compression=int(compression),
                      max_batch=int(max_batch), max_samples=int(max_samples),
-                     host_staging=int(bool(host_staging)), max_bank_samples=int(max_bank_samples))
+                     host_staging=int(bool(host_staging)), image_lattice=int(image_lattice),
+                     max_bank_samples=int(max_bank_samples))
 
 
 def aug_workspace_bytes(config: AugConfig) -> int:
@@ -157,6 +167,17 @@ def aug_sample_params(seed: int, dist: AugDist, lengths: np.ndarray, check: bool
     if check:
         _check(rc, "aug_sample_params")
     return rc, table
+
+
+def aug_bucket_by_length(lengths: np.ndarray, batch: int):
+    """(permutation by increasing length, longest length of each group of `batch`)."""
+    lengths = np.ascontiguousarray(lengths, dtype=np.int32)
+    B = int(lengths.shape[0])
+    perm = np.zeros(B, dtype=np.int32)
+    gmax = np.zeros(max(-(-B // int(batch)), 1), dtype=np.int32)
+    _check(lib().aug_bucket_by_length(lengths.ctypes.data, B, int(batch), perm.ctypes.data,
+                                      gmax.ctypes.data), "aug_bucket_by_length")
+    return perm, gmax[: -(-B // int(batch))]
 
 
 def aug_measure_fp32_peak(stream: Optional[int] = None) -> float:
@@ -290,6 +311,15 @@ class AugContext:
         return self._ret(lib().feat_vtlp_logmel(self._h, _ptr(power_dev), _ptr(counts_dev),
                                                 _ptr(table_dev), int(B), int(T_max),
                                                 _ptr(feats_dev)), "feat_vtlp_logmel", check)
+
+    def feat_mfcc(self, feats_dev, counts_dev, B, T_max, n_cep, mfcc_dev, check=True):
+        return self._ret(lib().feat_mfcc(self._h, _ptr(feats_dev), _ptr(counts_dev), int(B),
+                                         int(T_max), int(n_cep), _ptr(mfcc_dev)), "feat_mfcc", check)
+
+    def feat_mean_var(self, feats_dev, counts_dev, B, T_max, D, mean_dev, var_dev, check=True):
+        return self._ret(lib().feat_mean_var(self._h, _ptr(feats_dev), _ptr(counts_dev), int(B),
+                                             int(T_max), int(D), _ptr(mean_dev), _ptr(var_dev)),
+                         "feat_mean_var", check)
 
     def aug_pipeline(self, speech_dev, speech_stride, lengths_dev, lengths_host, bank_dev,
                      bank_len, table_dev, B, feats_dev, T_max, counts_dev, wave_out_dev=None,

@@ -26,6 +26,7 @@ int check_config(const AugConfig *c) {
     if (c->frac_half_width < 1 || c->frac_half_width > aug::MAX_HALF_W) return AUG_EINVAL;
     if (!(c->sound_speed > 0.f) || !(c->log_floor > 0.f) || !isfinite(c->pad_value)) return AUG_EINVAL;
     if (c->compression != AUG_COMPRESS_LOG && c->compression != AUG_COMPRESS_POW_1_15) return AUG_EINVAL;
+    if (c->image_lattice != AUG_LATTICE_TOTAL && c->image_lattice != AUG_LATTICE_CUBE) return AUG_EINVAL;
     if (c->max_batch < 1 || c->max_batch > 65535 || c->max_samples < 1) return AUG_EINVAL;
     if (c->host_staging && c->max_bank_samples < 0) return AUG_EINVAL;
     return AUG_OK;

@@ -23,7 +23,7 @@ __device__ __forceinline__ double ipow(double b, int e) {
 
 __global__ void __launch_bounds__(RIR_THREADS)
 rir_image_kernel(const AugUttParams *__restrict__ table, int S_max, int L, int half_w, double fs,
-                 double c, int max_order, float *__restrict__ rir, int *status) {
+                 double c, int max_order, int cube, float *__restrict__ rir, int *status) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     double *dsq = reinterpret_cast<double *>(smem_raw);   // [3][AX]
     double *gain = dsq + 3 * AX;                          // [3][AX]
@@ -69,7 +69,7 @@ rir_image_kernel(const AugUttParams *__restrict__ table, int S_max, int L, int h
         xpre[side] = run;
     }
     __syncthreads();
-    const int total = xpre[side];
+    const int total = cube ? side * side * side : xpre[side];
 
     // per-lane tap constants: this lane owns taps j = lane + 32 i - half_w
     float cj[3], sj[3], sg[3];
@@ -89,24 +89,32 @@ rir_image_kernel(const AugUttParams *__restrict__ table, int S_max, int L, int h
         int n0 = 0;
         float phi = 0.f, A = 0.f, As = 0.f, cph = 0.f, sph = 0.f;
         if (valid) {
-            // slab kx: the last ix with xpre[ix] <= idx
-            int lo = 0, hi = side;
-            while (hi - lo > 1) {
-                const int mid = (lo + hi) >> 1;
-                if (xpre[mid] <= idx) lo = mid; else hi = mid;
+            int ix, ky, kz;
+            if (cube) {
+                ix = idx / (side * side);
+                const int rem = idx - ix * side * side;
+                ky = rem / side - order;
+                kz = rem % side - order;
+            } else {
+                // slab kx: the last ix with xpre[ix] <= idx
+                int lo = 0, hi = side;
+                while (hi - lo > 1) {
+                    const int mid = (lo + hi) >> 1;
+                    if (xpre[mid] <= idx) lo = mid; else hi = mid;
+                }
+                ix = lo;
+                const int r = order - abs(ix - order);
+                int q = idx - xpre[ix];               // position inside the diamond of radius r
+                // rows ky = -r..0 hold 1, 3, .., 2r+1 points (q < (r+1)^2, row u has u^2 before it);
+                // rows ky = 1..r mirror rows r-1..0, counted from the end.
+                const bool upper = q >= (r + 1) * (r + 1);
+                if (upper) q = 2 * r * r + 2 * r - q;
+                int u = (int)sqrtf((float)q);
+                if (u * u > q) --u;
+                if ((u + 1) * (u + 1) <= q) ++u;
+                ky = upper ? r - u : u - r;
+                kz = q - u * u - u;
             }
-            const int ix = lo;
-            const int r = order - abs(ix - order);
-            int q = idx - xpre[ix];                   // position inside the diamond of radius r
-            // rows ky = -r..0 hold 1, 3, .., 2r+1 points (q < (r+1)^2, row u has u^2 before it);
-            // rows ky = 1..r mirror rows r-1..0, counted from the end.
-            const bool upper = q >= (r + 1) * (r + 1);
-            if (upper) q = 2 * r * r + 2 * r - q;
-            int u = (int)sqrtf((float)q);
-            if (u * u > q) --u;
-            if ((u + 1) * (u + 1) <= q) ++u;
-            const int ky = upper ? r - u : u - r;
-            const int kz = q - u * u - u;
             const int iy = ky + order, iz = kz + order;
             {
                 const double d = sqrt(dsq[ix] + dsq[AX + iy] + dsq[2 * AX + iz]);
@@ -165,7 +173,7 @@ int launch_rir(AugCtx *ctx, const AugUttParams *table, int B, float *rir, cudaSt
     dim3 grid(c.max_sources, B);
     rir_image_kernel<<<grid, RIR_THREADS, smem, st>>>(
         table, c.max_sources, c.rir_taps, c.frac_half_width, (double)c.fs, (double)c.sound_speed,
-        c.max_order, rir, ctx->status);
+        c.max_order, c.image_lattice == AUG_LATTICE_CUBE ? 1 : 0, rir, ctx->status);
     AUG_CUDA_OK(cudaGetLastError());
     ctx->launches++;
     return AUG_OK;

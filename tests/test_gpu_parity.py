@@ -44,6 +44,27 @@ def test_rir_matches_image_sum(index):
             assert err <= RIR_REL_TOL * np.max(np.abs(ref)), (index, b, s, err)
 
 
+def test_rir_distinct_walls_and_cube_lattice():
+    """Six different reflection coefficients (a swapped wall shows) and the cube lattice."""
+    w = small(2, batch=4, dur_scale=0.05, order=5)
+    rng = np.random.default_rng(3)
+    w.table["beta"] = rng.uniform(0.3, 0.95, (w.B, 6)).astype(np.float32)
+    for lattice, code in (("total", binding.LATTICE_TOTAL), ("cube", binding.LATTICE_CUBE)):
+        cfg = binding.make_config(w.cfg, w.B, w.stride, image_lattice=code)
+        ctx = binding.AugContext(cfg)
+        import torch
+        out = torch.full((w.B, cfg.max_sources, cfg.rir_taps), float("nan"), device="cuda")
+        ctx.aug_rir_image_method(binding.table_to_device(w.table), w.B, out)
+        torch.cuda.synchronize()
+        h = out.cpu().numpy()
+        for b in range(w.B):
+            row = w.table[b]
+            for s in range(int(row["n_src"])):
+                ref = oracle.rir_image_method(row["room"], row["beta"], row["mic"], row["src_pos"][s],
+                                              int(row["order"]), cfg.rir_taps, lattice=lattice)
+                assert np.max(np.abs(h[b, s] - ref)) <= RIR_REL_TOL * np.max(np.abs(ref)), (lattice, b, s)
+
+
 def test_rir_closed_form_single_image():
     w = small(1, batch=1, dur_scale=0.05)
     row = w.table[0]
@@ -201,3 +222,28 @@ def test_pipeline_runs_on_a_table_from_the_library_sampler():
         assert np.all(np.isfinite(F[b, :T])) and np.all(F[b, T:] == 0.0)
         assert np.all(np.isfinite(wave[b, : w.lengths[b]]))
         assert np.sqrt(np.mean(wave[b, : w.lengths[b]] ** 2)) > 1e-5
+
+
+def test_mfcc_and_mean_var_match():
+    import torch
+    w = small(5, **REDUCED[5])              # 128 mel bands, 1024-point FFT
+    w.lengths[0] = 300                      # an utterance without frames
+    dev = Device(w)
+    F, counts, _ = dev.pipeline(want_wave=False)
+    n_cep = 20
+    C = torch.full((w.B, dev.T_max, n_cep), float("nan"), device="cuda")
+    dev.ctx.feat_mfcc(F, counts, w.B, dev.T_max, n_cep, C)
+    mean = torch.full((w.B, dev.M), float("nan"), device="cuda")
+    var = torch.full((w.B, dev.M), float("nan"), device="cuda")
+    dev.ctx.feat_mean_var(F, counts, w.B, dev.T_max, dev.M, mean, var)
+    torch.cuda.synchronize()
+    Fh, Ch, ch = F.cpu().numpy().astype(np.float64), C.cpu().numpy(), counts.cpu().numpy()
+    for b in range(w.B):
+        T = int(ch[b])
+        ref = oracle.mfcc(Fh[b, :T], n_cep)
+        assert np.max(np.abs(Ch[b, :T] - ref), initial=0.0) <= 1e-4 * max(1.0, np.max(np.abs(ref), initial=0.0))
+        assert np.all(Ch[b, T:] == w.cfg["pad_value"])
+        mu, vr = oracle.mean_var(Fh[b, :T])
+        np.testing.assert_allclose(mean[b].cpu().numpy(), mu, atol=1e-5 * (1 + np.max(np.abs(mu))))
+        np.testing.assert_allclose(var[b].cpu().numpy(), vr, atol=1e-4 * (1 + np.max(np.abs(vr))))
+    assert dev.ctx.feat_mfcc(F, counts, w.B, dev.T_max, dev.M + 1, C, check=False) == binding.AUG_EINVAL

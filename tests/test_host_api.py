@@ -143,6 +143,20 @@ def test_sample_params_rejects_bad_ranges():
     assert binding.aug_sample_params(0, _dist(bank_len=0), lengths, check=False)[0] == binding.AUG_EINVAL
 
 
+def test_bucket_by_length():
+    lengths = np.array([500, 100, 300, 100, 900, 200, 700], dtype=np.int32)
+    perm, gmax = binding.aug_bucket_by_length(lengths, 3)
+    assert list(perm) == [1, 3, 5, 2, 0, 6, 4]            # increasing length, ties in input order
+    assert list(gmax) == [200, 700, 900]
+    rng = np.random.default_rng(0)
+    lengths = rng.integers(16000, 320000, 256).astype(np.int32)
+    perm, gmax = binding.aug_bucket_by_length(lengths, 16)
+    assert sorted(perm) == list(range(256))
+    padded_sorted = int(np.sum(gmax.astype(np.int64) * 16))
+    padded_plain = int(sum(lengths[i:i + 16].max() * 16 for i in range(0, 256, 16)))
+    assert padded_sorted < 0.65 * padded_plain and padded_sorted >= int(lengths.sum())
+
+
 def test_compute_calls_refuse_without_a_gpu():
     import torch
     if torch.cuda.is_available():

@@ -21,6 +21,7 @@ PIN_CALLS = [
     lambda: pins.test_rir_matches_mirror_construction_at_low_frequency(1),
     lambda: pins.test_rir_matches_mirror_construction_at_low_frequency(3),
     pins.test_rir_reciprocity,
+    lambda: pins.test_rir_cube_lattice_count_and_mirror_construction(1),
     pins.test_fractional_delay_kernel_delays_a_sinusoid,
     pins.test_delay_kernel_window_shape,
     pins.test_rir_taps_outside_the_buffer_are_dropped,
@@ -68,7 +69,8 @@ C_MUTATIONS = {
                                      "(1 - 2 * p) * src[a] + 2.0 * (m - p) * room[a]"),
     "delay kernel window too wide": ("cos(M_PI * x / half_w)", "cos(M_PI * x / (half_w + 8))"),
     "delay sign": ("double x = (double)n - tau;", "double x = (double)n + 1.0 - tau;"),
-    "L-infinity order": ("if (abs(kx) + abs(ky) + abs(kz) > order) continue;", ""),
+    "L-infinity order": ("if (!cube && abs(kx) + abs(ky) + abs(kz) > order) continue;", ""),
+    "cube flag ignored": ("if (!cube && abs(kx)", "if (abs(kx)"),
     "last tap dropped": ("int64_t jmax = n < L - 1 ? n : L - 1;", "int64_t jmax = n < L - 2 ? n : L - 2;"),
     "symmetric Hann": ("0.5 - 0.5 * cos(2.0 * M_PI * n / win)", "0.5 - 0.5 * cos(2.0 * M_PI * n / (win - 1))"),
     "frame count rounds up": ("return (int)(1 + (N - win) / hop);", "return (int)(1 + (N - win + hop - 1) / hop);"),

@@ -39,7 +39,32 @@ def test_rir_image_count(order):
     assert n == (2 * order + 1) * (2 * order * order + 2 * order + 3) // 3
 
 
-def _mirror_images(room, beta, src, order):
+@pytest.mark.parametrize("order", [0, 1, 3])
+def test_rir_cube_lattice_count_and_mirror_construction(order):
+    room, mic, src = [3.1, 2.7, 2.4], [1.0, 1.3, 1.1], [2.2, 0.9, 1.6]
+    beta = [0.9, 0.5, 0.8, 0.4, 0.7, 0.3]
+    L = 2048
+    h, n = oracle.rir_image_method(room, beta, mic, src, order, L, return_count=True, lattice="cube")
+    assert n == (2 * order + 1) ** 3
+    imgs = _mirror_images(room, beta, src, order, cube=True)
+    assert len(imgs) == n
+    f = np.array([50.0, 230.0, 700.0, 1500.0, 2900.0])
+    k = np.arange(L)
+    H = np.array([np.sum(h * np.exp(-2j * np.pi * fi / FS * k)) for fi in f])
+    ref = np.zeros_like(H)
+    scale = 0.0
+    for pos, g in imgs:
+        d = np.linalg.norm(np.array(pos) - np.array(mic))
+        if d * FS / C + 40 < L:                          # later images fall outside the buffer
+            ref += (g / d) * np.exp(-2j * np.pi * f * d / C)
+        scale += g / d
+    assert np.max(np.abs(H - ref)) < 2e-3 * scale
+    if order:
+        total = oracle.rir_image_method(room, beta, mic, src, order, L)
+        assert np.max(np.abs(h - total)) > 1e-4          # the cube really holds more images
+
+
+def _mirror_images(room, beta, src, order, cube=False):
     """All image sources up to `order` reflections, built by composing mirror
     reflections in the real walls (x -> -x at the wall at 0, x -> 2L - x at the wall
     at L), walls alternating along an axis.  Independent of the k = 2m - p indexing."""
@@ -57,7 +82,7 @@ def _mirror_images(room, beta, src, order):
         per_axis.append(opts)
     out = []
     for (nx, x, gx), (ny, y, gy), (nz, z, gz) in itertools.product(*per_axis):
-        if nx + ny + nz <= order:
+        if cube or nx + ny + nz <= order:
             out.append(((x, y, z), gx * gy * gz))
     return out
 
@@ -357,3 +382,26 @@ def test_delta_rir_path_returns_the_input_features():
     ref = oracle.logmel(oracle.stft_power(np.concatenate([np.zeros(lag), x[:-lag]]) / d,
                                           400, 160, 512), 1.0, 512, 40, floor=cfg["log_floor"])
     np.testing.assert_allclose(out["feats"], ref, atol=1e-9)
+
+
+# ------------------------------------------------------------------ after the features
+def test_mfcc_is_the_orthonormal_dct():
+    import scipy.fft
+    x = np.random.default_rng(21).standard_normal((7, 40))
+    np.testing.assert_allclose(oracle.mfcc(x, 40), scipy.fft.dct(x, type=2, norm="ortho", axis=1),
+                               atol=1e-12)
+    np.testing.assert_allclose(oracle.mfcc(x, 13), scipy.fft.dct(x, type=2, norm="ortho", axis=1)[:, :13],
+                               atol=1e-12)
+    c = oracle.mfcc(np.full((1, 40), 2.5), 40)          # a flat spectrum has only c_0 = sqrt(M) x
+    assert c[0, 0] == pytest.approx(2.5 * np.sqrt(40)) and np.max(np.abs(c[0, 1:])) < 1e-12
+    assert np.sum(oracle.mfcc(x, 40) ** 2) == pytest.approx(np.sum(x ** 2))   # orthonormal
+
+
+def test_mean_var_closed_forms():
+    t = np.arange(101.0)
+    x = np.stack([t, np.full(101, 3.0), (-1.0) ** t], axis=1)
+    mu, var = oracle.mean_var(x)
+    np.testing.assert_allclose(mu, [50.0, 3.0, 1 / 101], atol=1e-12)
+    np.testing.assert_allclose(var, [(101 ** 2 - 1) / 12, 0.0, 1 - (1 / 101) ** 2], atol=1e-9)
+    mu, var = oracle.mean_var(np.zeros((0, 5)))
+    assert not mu.any() and not var.any()
