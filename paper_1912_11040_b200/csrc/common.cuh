@@ -16,7 +16,10 @@ constexpr int MAX_HALF_W = 47;
 constexpr int MAX_MEL = 128;
 
 constexpr int EV_RING = 256;
-constexpr int HOST_CHUNKS = 8;           // pipeline depth of aug_pipeline_host
+#ifndef AUG_HOST_CHUNKS
+#define AUG_HOST_CHUNKS 8
+#endif
+constexpr int HOST_CHUNKS = AUG_HOST_CHUNKS;   // pipeline depth of aug_pipeline_host
 
 enum Reason { R_NONE = 0, R_NSRC = 1, R_ORDER = 2, R_NOISE = 3, R_WAIT = 4 };
 
