@@ -35,15 +35,20 @@ SM_COUNT, FP32_LANES = 148, 128
 # DRAM bytes per audio-second of workload 2 (dram__bytes_read.sum + dram__bytes_write.sum of one
 # ncu --set full capture on 96 utterances; traffic grows in proportion to the audio processed).
 # Valid only for the kernel sources the capture was taken from: the hash guards that.
-NCU_TRAFFIC = {"workload": 2, "sources_sha": "f7eb0b1a28015847",
-               "bytes_per_audio_s": {"convolve": 466.58e6 / 1039.18, "block_spectra": 403.27e6 / 1039.18,
-                                     "features": 148.79e6 / 1039.18, "rir_image": 0.04e6 / 1039.18}}
+NCU_TRAFFIC = {
+    "workload": 2,
+    "bytes_per_audio_s": {"convolve": 466.58e6 / 1039.18, "block_spectra": 403.27e6 / 1039.18,
+                          "features": 148.79e6 / 1039.18},
+    # kernel -> (its source files, sha256[:16] of them when the counters were taken)
+    "sources": {"convolve": (("conv.cu", "fft.cuh"), "deae2bb07dd8de72"),
+                "block_spectra": (("conv.cu", "fft.cuh"), "deae2bb07dd8de72"),
+                "features": (("feat.cu", "fft.cuh"), "51443e66ec633c23")}}
 
 
-def kernel_sources_sha():
+def kernel_sources_sha(files):
     import hashlib
     h = hashlib.sha256()
-    for f in ("conv.cu", "fft.cuh", "feat.cu", "rir.cu"):
+    for f in files:
         h.update(open(os.path.join(ROOT, "paper_1912_11040_b200", "csrc", f), "rb").read())
     return h.hexdigest()[:16]
 
@@ -365,7 +370,7 @@ def run_ours(args):
                     "unit": "GB/s", "frac": d["frac_hbm"], "traffic": None,
                     "peak_source": f"{hbm_src} copy bandwidth"}
     if (args.workload == NCU_TRAFFIC["workload"] and dom in NCU_TRAFFIC["bytes_per_audio_s"]
-            and kernel_sources_sha() == NCU_TRAFFIC["sources_sha"]):
+            and kernel_sources_sha(NCU_TRAFFIC["sources"][dom][0]) == NCU_TRAFFIC["sources"][dom][1]):
         roofline["traffic"] = NCU_TRAFFIC["bytes_per_audio_s"][dom] * w.audio_seconds
         roofline["traffic_note"] = ("bytes per launch, ncu capture on 96 utterances scaled by audio-seconds; "
                                     "algorithmic bytes of this kernel: %.3e" % kernels[dom][1][1])
