@@ -247,3 +247,44 @@ def test_mfcc_and_mean_var_match():
         np.testing.assert_allclose(mean[b].cpu().numpy(), mu, atol=1e-5 * (1 + np.max(np.abs(mu))))
         np.testing.assert_allclose(var[b].cpu().numpy(), vr, atol=1e-4 * (1 + np.max(np.abs(vr))))
     assert dev.ctx.feat_mfcc(F, counts, w.B, dev.T_max, dev.M + 1, C, check=False) == binding.AUG_EINVAL
+
+
+def test_empty_batch_is_a_no_op():
+    w = small(1, batch=1, dur_scale=0.1)
+    dev = Device(w)
+    import torch
+    F = torch.full((1, dev.T_max, dev.M), 7.0, device="cuda")
+    c = torch.full((1,), 7, dtype=torch.int32, device="cuda")
+    assert dev.ctx.aug_pipeline(dev.speech, w.stride, dev.lengths, None, dev.bank, w.bank.size,
+                                dev.table, 0, F, dev.T_max, c, check=False) == binding.AUG_OK
+    torch.cuda.synchronize()
+    assert float(F.min()) == 7.0 and int(c[0]) == 7
+
+
+def test_pipeline_at_the_configuration_limits():
+    """Largest reflection order, tap count, delay-kernel width, band count and source
+    count a context accepts, on one short utterance."""
+    w = small(5, batch=1, dur_scale=1.0 / 60.0, taps=24576, order=32)     # 1 s, 1024-point FFT, 128 mel
+    w.cfg["frac_half_width"] = 47
+    row = w.table[0]
+    rng = np.random.default_rng(9)
+    row["n_src"] = 4
+    row["beta"] = rng.uniform(0.6, 0.97, 6)
+    for s in range(1, 4):
+        row["src_pos"][s] = [rng.uniform(0.4, float(row["room"][a]) - 0.4) for a in range(3)]
+    n = int(w.lengths[0])
+    for k in range(3):
+        row["noise_len"][k] = 5000 + 1111 * k
+        row["noise_offset"][k] = 1000 * (k + 1)
+        row["noise_weight"][k] = 0.5 + 0.5 * k
+    dev = Device(w)
+    assert binding.aug_validate_params(dev.cfg, w.table, w.bank.size) == (0, -1)
+    F, counts, wave = dev.pipeline(want_wave=True)
+    assert dev.ctx.aug_last_status() == (-1, 0)
+    worst_f, worst_w = check_pipeline_against_oracle(dev, F, counts, wave, oracle_batch(w))
+    print(f"limits: worst log-mel err {worst_f:.2e}, worst wave err/rms {worst_w:.2e}")
+    # one step beyond each limit is refused when the context is created
+    for field, value in [("max_order", 33), ("rir_taps", 24577), ("frac_half_width", 48), ("n_mel", 129)]:
+        cfg = binding.make_config(dict(w.cfg, **{field: value}), 1, w.stride)
+        with pytest.raises(binding.AugError):
+            binding.AugContext(cfg)
