@@ -187,6 +187,108 @@ def time_oracle(w, budget_s, max_seconds_per_utt=None):
     return done_audio / dt, f"first {n_utt} utterance(s), {done_audio:.1f} audio-s, {dt:.1f} s wall", cores
 
 
+# ------------------------------------------------------------------ fast CPU pipeline
+# A reasonable CPU implementation of the same four steps (vectorised image sum, FFT
+# convolution, rfft STFT, dense mel matrix; numpy/scipy, fp64), one process per core:
+# the stand-in for the paper's CPU example servers.  Context for the GPU number only;
+# it shares nothing with the CUDA library or the fp64 checker.
+_LATTICE = {}
+
+
+def _fast_lattice(order):
+    if order not in _LATTICE:
+        k = np.arange(-order, order + 1)
+        kx, ky, kz = np.meshgrid(k, k, k, indexing="ij")
+        keep = (np.abs(kx) + np.abs(ky) + np.abs(kz)) <= order
+        _LATTICE[order] = np.stack([kx[keep], ky[keep], kz[keep]], axis=1)
+    return _LATTICE[order]
+
+
+def _fast_rir(row, s, cfg):
+    L, hw, fs, c = int(cfg["rir_taps"]), int(cfg["frac_half_width"]), float(cfg["fs"]), float(cfg["sound_speed"])
+    k = _fast_lattice(int(row["order"]))
+    p = k & 1
+    m = (k + p) // 2
+    room, src, mic = (np.asarray(row[n], dtype=np.float64) for n in ("room", "src_pos", "mic"))
+    img = (1 - 2 * p) * src[s] + 2.0 * m * room
+    d = np.sqrt(((img - mic) ** 2).sum(axis=1))
+    beta = np.asarray(row["beta"], dtype=np.float64)
+    gain = np.prod(beta[0::2] ** np.abs(m - p) * beta[1::2] ** np.abs(m), axis=1)
+    tau = d * fs / c
+    n0 = np.rint(tau).astype(np.int64)
+    idx = n0[:, None] + np.arange(-hw, hw + 1)[None, :]
+    x = idx - tau[:, None]
+    val = (gain / d)[:, None] * np.sinc(x) * 0.5 * (1.0 + np.cos(np.pi * x / hw))
+    ok = (idx >= 0) & (idx < L) & (np.abs(x) <= hw)
+    return np.bincount(idx[ok], weights=val[ok], minlength=L)[:L]
+
+
+def _fast_mel(alpha, cfg):
+    K, M, fs = int(cfg["n_fft"]), int(cfg["n_mel"]), float(cfg["fs"])
+    w = 2.0 * np.pi * np.arange(K // 2 + 1) / K
+    a = 1.0 - float(alpha)
+    fw = (w + 2.0 * np.arctan(a * np.sin(w) / (1.0 - a * np.cos(w)))) * fs / (2.0 * np.pi)
+    mel = lambda f: 2595.0 * np.log10(1.0 + f / 700.0)
+    e = np.linspace(mel(float(cfg["f_lo"])), mel(float(cfg["f_hi"])), M + 2)
+    mu = mel(fw)[None, :]
+    up = (mu - e[:-2, None]) / (e[1:-1, None] - e[:-2, None])
+    dn = (e[2:, None] - mu) / (e[2:, None] - e[1:-1, None])
+    return np.maximum(0.0, np.minimum(up, dn))
+
+
+def fast_cpu_utterance(speech, bank, row, cfg):
+    """Log-mel features [T][M] of one utterance, fp64 numpy/scipy."""
+    from scipy.signal import fftconvolve
+    n = len(speech)
+    ys = fftconvolve(np.asarray(speech, dtype=np.float64), _fast_rir(row, 0, cfg))[:n]
+    out = ys
+    if int(row["n_src"]) > 1:
+        v = np.zeros(n)
+        for j in range(int(row["n_src"]) - 1):
+            seg = np.asarray(bank[int(row["noise_offset"][j]): int(row["noise_offset"][j]) + int(row["noise_len"][j])],
+                             dtype=np.float64)
+            v += float(row["noise_weight"][j]) * fftconvolve(np.resize(seg, n), _fast_rir(row, 1 + j, cfg))[:n]
+        es, ev = float(ys @ ys), float(v @ v)
+        if es > 0 and ev > 0:
+            out = ys + np.sqrt(es / (ev * 10.0 ** (float(row["snr_db"]) / 10.0))) * v
+    W, H, K = int(cfg["win"]), int(cfg["hop"]), int(cfg["n_fft"])
+    if n < W:
+        return np.zeros((0, int(cfg["n_mel"])))
+    T = 1 + (n - W) // H
+    frames = np.lib.stride_tricks.as_strided(out, (T, W), (out.strides[0] * H, out.strides[0]))
+    P = np.abs(np.fft.rfft(frames * (0.5 - 0.5 * np.cos(2.0 * np.pi * np.arange(W) / W)), K, axis=1)) ** 2
+    return np.log(np.maximum(P @ _fast_mel(row["alpha"], cfg).T, float(cfg["log_floor"])))
+
+
+def _fast_worker(job):
+    speech_rows, lengths, bank, table, cfg = job
+    t0 = time.perf_counter()
+    for b in range(len(lengths)):
+        fast_cpu_utterance(speech_rows[b][: lengths[b]], bank, table[b], cfg)
+    return float(sum(lengths)) / cfg["fs"], time.perf_counter() - t0
+
+
+def time_fast_cpu(w, n_utts):
+    """The first n_utts utterances through fast_cpu_utterance, spread over all cores
+    (spawned workers).  Returns (audio-s/s, description, workers)."""
+    import multiprocessing as mp
+    workers = max(1, min(os.cpu_count() or 1, n_utts))
+    n_utts = min(n_utts, w.B)
+    jobs = []
+    for k in range(workers):
+        sel = list(range(k, n_utts, workers))
+        if sel:
+            jobs.append(([w.speech[b, : w.lengths[b]].copy() for b in sel], [int(w.lengths[b]) for b in sel],
+                         w.bank, w.table[sel].copy(), dict(w.cfg)))
+    with mp.get_context("spawn").Pool(len(jobs)) as pool:
+        pool.map(_fast_worker, [(j[0][:1], j[1][:1], j[2], j[3][:1], j[4]) for j in jobs])   # start-up, imports
+        t0 = time.perf_counter()
+        res = pool.map(_fast_worker, jobs)
+        dt = time.perf_counter() - t0
+    audio = sum(r[0] for r in res)
+    return audio / dt, f"first {n_utts} utterance(s), {audio:.1f} audio-s, {dt:.1f} s wall, numpy/scipy fp64", len(jobs)
+
+
 def run_reference(args):
     """The CPU checker as the reference arm: each step is one utterance of the
     workload (cut to 5 s) through all four steps in fp64 on the host cores."""
@@ -397,6 +499,10 @@ def run_ours(args):
             "roofline": roofline,
             "cpu_baseline": {"value": cpu_val, "unit": UNIT, "cores": cores, "kind": "oracle",
                              "sample": cpu_sample}}
+    if args.cpu_fast_utts > 0:
+        fv, fs_, fw = time_fast_cpu(w, args.cpu_fast_utts)
+        line["cpu_fast"] = {"value": fv, "unit": UNIT, "cores": fw, "kind": "numpy/scipy FFT pipeline",
+                            "sample": fs_}
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -412,6 +518,8 @@ def main():
     ap.add_argument("--workload", type=int, default=2, choices=[1, 2, 3, 4, 5])
     ap.add_argument("--cpu-budget", type=float, default=15.0,
                     help="seconds of wall time given to the CPU-checker baseline")
+    ap.add_argument("--cpu-fast-utts", type=int, default=64,
+                    help="utterances given to the numpy/scipy CPU pipeline (0 = skip)")
     ap.add_argument("--batch", type=int, default=None,
                     help="profiling runs: fewer utterances than the workload's own batch")
     ap.add_argument("--skip-e2e", action="store_true",
