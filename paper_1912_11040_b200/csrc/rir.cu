@@ -12,7 +12,10 @@
 
 namespace {
 
-constexpr int RIR_THREADS = 512;
+#ifndef RIR_THREADS_N
+#define RIR_THREADS_N 1024
+#endif
+constexpr int RIR_THREADS = RIR_THREADS_N;
 constexpr int AX = 2 * aug::MAX_ORDER + 1;
 
 __device__ __forceinline__ double ipow(double b, int e) {
@@ -146,7 +149,7 @@ rir_image_kernel(const AugUttParams *__restrict__ table, int S_max, int L, int h
                 const int j = jj - half_w;
                 const int n = n0b + j;
                 const float x = (float)j - phib;
-                if (jj <= 2 * half_w && n >= 0 && n < L && fabsf(x) <= fhw) {
+                if (jj <= 2 * half_w && (unsigned)n < (unsigned)L && fabsf(x) <= fhw) {
                     const float hann = 0.5f + cj[i] * cb + sj[i] * sb;
                     const float sc = (fabsf(x) < 1e-7f) ? Ab : __fdividef(sg[i] * Asb, x);
                     atomicAdd(&h[n], sc * hann);
