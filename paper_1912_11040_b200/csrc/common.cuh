@@ -51,6 +51,7 @@ struct AugCtx {
     float *ys;             // [max_batch][ws_stride]
     float *vv;             // [max_batch][ws_stride]
     double *energy;        // [max_batch][2]
+    float *gain;           // [max_batch] noise gain g for the requested SNR
     aug::MelBin *melw;     // [max_batch][n_bins]
     int *melstart;         // [max_batch][n_mel + 2]
     int *status;           // [2]: utterance, reason

@@ -386,22 +386,29 @@ spectral_convolve_kernel(const int *__restrict__ lengths, const float *__restric
 }
 
 // ---------------------------------------------------------------- mixing
-__device__ __forceinline__ float snr_gain(const double *energy, int utt, int n_src, float snr_db) {
+// g = sqrt(sum y_s^2 / (sum v^2 10^(snr/10))), 0 without noise or with a silent side:
+// once per utterance, in fp64, after the convolution has finished the two sums.
+__global__ void __launch_bounds__(256)
+snr_gain_kernel(const double *__restrict__ energy, const AugUttParams *__restrict__ table, int B,
+                float *__restrict__ gain) {
+    const int utt = blockIdx.x * 256 + threadIdx.x;
+    if (utt >= B) return;
     const double es = energy[2 * utt], ev = energy[2 * utt + 1];
-    if (n_src <= 1 || !(es > 0.0) || !(ev > 0.0)) return 0.f;
-    return (float)sqrt(es / (ev * pow(10.0, (double)snr_db / 10.0)));
+    float g = 0.f;
+    if (table[utt].n_src > 1 && es > 0.0 && ev > 0.0)
+        g = (float)sqrt(es / (ev * pow(10.0, (double)table[utt].snr_db / 10.0)));
+    gain[utt] = g;
 }
 
 __global__ void __launch_bounds__(256)
 mix_kernel(const float *__restrict__ ys, const float *__restrict__ vv, int64_t ws_stride,
-           const double *__restrict__ energy, const int *__restrict__ lengths,
-           const AugUttParams *__restrict__ table, float *__restrict__ out, int64_t out_stride,
-           int n_cap) {
+           const float *__restrict__ gain, const int *__restrict__ lengths,
+           float *__restrict__ out, int64_t out_stride, int n_cap) {
     const int utt = blockIdx.y;
     const int N = min(max(lengths[utt], 0), n_cap);
     const int i = (blockIdx.x * 256 + threadIdx.x) * 4;
     if (i >= N) return;
-    const float g = snr_gain(energy, utt, table[utt].n_src, table[utt].snr_db);
+    const float g = gain[utt];
     const float *a = ys + (int64_t)utt * ws_stride + i;
     const float *b = vv + (int64_t)utt * ws_stride + i;
     float *o = out + (int64_t)utt * out_stride + i;
@@ -467,6 +474,9 @@ int launch_convolve_finish(AugCtx *ctx, const float *speech, int64_t stride, con
     }
     AUG_CUDA_OK(cudaGetLastError());
     ctx->launches++;
+    snr_gain_kernel<<<(B + 255) / 256, 256, 0, ctx->stream>>>(ctx->energy, table, B, ctx->gain);
+    AUG_CUDA_OK(cudaGetLastError());
+    ctx->launches++;
     return AUG_OK;
 }
 
@@ -474,8 +484,8 @@ int launch_mix(AugCtx *ctx, const int *lengths, const AugUttParams *table, int B
                float *wave_out, int64_t out_stride) {
     if (max_len <= 0) return AUG_OK;
     dim3 grid((max_len + 1023) / 1024, B);
-    mix_kernel<<<grid, 256, 0, ctx->stream>>>(ctx->ys, ctx->vv, ctx->ws_stride, ctx->energy, lengths,
-                                              table, wave_out, out_stride, max_len);
+    mix_kernel<<<grid, 256, 0, ctx->stream>>>(ctx->ys, ctx->vv, ctx->ws_stride, ctx->gain, lengths,
+                                              wave_out, out_stride, max_len);
     AUG_CUDA_OK(cudaGetLastError());
     ctx->launches++;
     return AUG_OK;

@@ -167,17 +167,11 @@ struct Plan<1024> {
     static constexpr int E = 16, FT = FEAT_FT_1024;
 };
 
-__device__ __forceinline__ float snr_gain_f(const double *energy, int utt, int n_src, float snr_db) {
-    const double es = energy[2 * utt], ev = energy[2 * utt + 1];
-    if (n_src <= 1 || !(es > 0.0) || !(ev > 0.0)) return 0.f;
-    return (float)sqrt(es / (ev * pow(10.0, (double)snr_db / 10.0)));
-}
-
 // MODE 0: wave -> power (global).  MODE 1: y_s + g v -> features.
 template <int K, int MODE>
 __global__ void __launch_bounds__(FEAT_THREADS)
 frames_kernel(const float *__restrict__ in_a, const float *__restrict__ in_b, int64_t in_stride,
-              const double *__restrict__ energy, const AugUttParams *__restrict__ table,
+              const float *__restrict__ gain, const AugUttParams *__restrict__ table,
               const int *__restrict__ lengths, int win, int hop, int M, int T_max,
               const aug::MelBin *__restrict__ melw, const int *__restrict__ melstart,
               const float2 *__restrict__ tw, float floor_v, float pad_v, int comp,
@@ -209,7 +203,7 @@ frames_kernel(const float *__restrict__ in_a, const float *__restrict__ in_b, in
     const int ns = (nf - 1) * hop + win;
     const float *pa = in_a + (int64_t)utt * in_stride + s0;
     if (MODE == 1) {
-        const float g = snr_gain_f(energy, utt, table[utt].n_src, table[utt].snr_db);
+        const float g = gain[utt];
         const float *pb = in_b + (int64_t)utt * in_stride + s0;
         if ((hop & 3) == 0) {
             for (int i = tid * 4; i < ns; i += FEAT_THREADS * 4) {
@@ -305,7 +299,7 @@ int launch_frames(AugCtx *ctx, const float *a, const float *b, int64_t stride, c
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     dim3 grid((T_max + FT - 1) / FT, B);
     frames_kernel<K, MODE><<<grid, FEAT_THREADS, smem, ctx->stream>>>(
-        a, b, stride, ctx->energy, table, lengths, c.win, c.hop, c.n_mel, T_max, ctx->melw,
+        a, b, stride, ctx->gain, table, lengths, c.win, c.hop, c.n_mel, T_max, ctx->melw,
         ctx->melstart, ctx->tw, c.log_floor, c.pad_value, c.compression, out, counts,
         (int)(stride < 0x7fffffff ? stride : 0x7fffffff));
     AUG_CUDA_OK(cudaGetLastError());
