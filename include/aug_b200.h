@@ -157,8 +157,9 @@ int aug_destroy(AugCtx *ctx);
 
 /* Synchronises the context's stream and reads the device status word.
  * *utt_host = first utterance a kernel rejected (-1 if none), *reason_host =
- * 1 n_src out of range, 2 order out of range, 3 bad noise stretch, 4 a bounded
- * wait inside a kernel ran out.  A rejected utterance gets zero impulse
+ * 1 n_src out of range, 2 order out of range, 3 bad noise stretch (the kernels
+ * contain no waits on other blocks, so nothing else can go wrong on the device
+ * short of a launch failure).  A rejected utterance gets zero impulse
  * responses / silent output; nothing faults.  The word is cleared by the read. */
 int aug_last_status(AugCtx *ctx, int *utt_host, int *reason_host);
 

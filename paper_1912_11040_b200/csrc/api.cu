@@ -37,7 +37,7 @@ struct Layout {
     int64_t ws_stride;
     int64_t off_xspec;
     int64_t off_tw, off_rir, off_hspec, off_ys, off_vv, off_energy, off_gain, off_melw, off_melstart,
-        off_status, off_counts, off_st_speech, off_st_bank, off_st_table, off_st_lengths,
+        off_status, off_st_speech, off_st_bank, off_st_table, off_st_lengths,
         off_st_feats, off_st_counts, total;
 };
 
@@ -62,7 +62,6 @@ Layout make_layout(const AugConfig &c) {
     l.off_melw = take(sizeof(aug::MelBin) * B * l.n_bins);
     l.off_melstart = take(sizeof(int) * B * (c.n_mel + 2));
     l.off_status = take(sizeof(int) * 2);
-    l.off_counts = take(sizeof(int) * B);
     if (c.host_staging) {
         l.off_st_speech = take(sizeof(float) * B * l.ws_stride);
         l.off_st_bank = take(sizeof(float) * (c.max_bank_samples > 0 ? c.max_bank_samples : 1));
@@ -184,7 +183,6 @@ int aug_create(AugCtx **out, const AugConfig *cfg, void *cuda_stream) {
     ctx->melw = reinterpret_cast<aug::MelBin *>(base + l.off_melw);
     ctx->melstart = reinterpret_cast<int *>(base + l.off_melstart);
     ctx->status = reinterpret_cast<int *>(base + l.off_status);
-    ctx->counts_tmp = reinterpret_cast<int *>(base + l.off_counts);
     if (cfg->host_staging) {
         ctx->st_speech = reinterpret_cast<float *>(base + l.off_st_speech);
         ctx->st_bank = reinterpret_cast<float *>(base + l.off_st_bank);
@@ -378,8 +376,7 @@ int aug_pipeline(AugCtx *ctx, const float *speech_dev, int64_t speech_stride,
         return rc;
     t1(5, sm);
     t0(6, sm);
-    rc = launch_fused_features(ctx, lengths_dev, table_dev, B, feats_dev, T_max, frame_counts_dev,
-                               nullptr, 0);
+    rc = launch_fused_features(ctx, lengths_dev, table_dev, B, feats_dev, T_max, frame_counts_dev);
     t1(6, sm);
     if (ev && rc == AUG_OK) ctx->ev_n++;
     return rc;

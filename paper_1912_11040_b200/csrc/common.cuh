@@ -21,7 +21,7 @@ constexpr int EV_RING = 256;
 #endif
 constexpr int HOST_CHUNKS = AUG_HOST_CHUNKS;   // pipeline depth of aug_pipeline_host
 
-enum Reason { R_NONE = 0, R_NSRC = 1, R_ORDER = 2, R_NOISE = 3, R_WAIT = 4 };
+enum Reason { R_NONE = 0, R_NSRC = 1, R_ORDER = 2, R_NOISE = 3 };
 
 // Per-bin entry of the warped filterbank: the bin lies in edge interval `seg`
 // (between edges e_seg and e_seg+1), at fraction `up` from its lower edge.
@@ -55,7 +55,6 @@ struct AugCtx {
     aug::MelBin *melw;     // [max_batch][n_bins]
     int *melstart;         // [max_batch][n_mel + 2]
     int *status;           // [2]: utterance, reason
-    int *counts_tmp;       // [max_batch]
     // instrumentation
     int64_t launches;      // kernels launched so far
     int timing;            // record events between the stages of aug_pipeline
@@ -101,5 +100,4 @@ int launch_stft_power(AugCtx *ctx, const float *wave, int64_t stride, const int 
 int launch_logmel(AugCtx *ctx, const float *power, const int *counts, int B, int T_max,
                   float *feats);
 int launch_fused_features(AugCtx *ctx, const int *lengths, const AugUttParams *table, int B,
-                          float *feats, int T_max, int *counts, float *wave_out,
-                          int64_t out_stride);
+                          float *feats, int T_max, int *counts);

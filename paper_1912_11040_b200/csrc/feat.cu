@@ -328,7 +328,7 @@ int launch_stft_power(AugCtx *ctx, const float *wave, int64_t stride, const int 
 }
 
 int launch_fused_features(AugCtx *ctx, const int *lengths, const AugUttParams *table, int B,
-                          float *feats, int T_max, int *counts, float *, int64_t) {
+                          float *feats, int T_max, int *counts) {
     if (T_max <= 0) return AUG_OK;
     if (ctx->cfg.n_fft == 512)
         return launch_frames<512, 1>(ctx, ctx->ys, ctx->vv, ctx->ws_stride, lengths, table, B, feats,
