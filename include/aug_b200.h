@@ -25,6 +25,9 @@
  *     recorded in a device status word, see aug_last_status.
  *   - Audio is fp32 at AugConfig.fs; sample counts and frame counts are int32;
  *     offsets into the noise bank are int64.
+ *   - A context serialises its work on its one stream and reuses one workspace:
+ *     use it from one host thread at a time; several contexts (one per thread or
+ *     per stream) are independent.  Use a context on the device it was created on.
  */
 #ifndef AUG_B200_H
 #define AUG_B200_H

@@ -166,13 +166,9 @@ rir_image_kernel(const AugUttParams *__restrict__ table, int S_max, int L, int h
 int launch_rir(AugCtx *ctx, const AugUttParams *table, int B, float *rir, cudaStream_t st) {
     const AugConfig &c = ctx->cfg;
     const size_t smem = sizeof(double) * 6 * AX + sizeof(int) * (AX + 3) + sizeof(float) * (size_t)c.rir_taps;
-    static bool attr_set = false;
-    if (!attr_set) {
-        AUG_CUDA_OK(cudaFuncSetAttribute(rir_image_kernel,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)(sizeof(double) * 6 * AX + sizeof(int) * (AX + 3) + sizeof(float) * aug::MAX_TAPS)));
-        attr_set = true;
-    }
+    // (set on every launch: the attribute belongs to the current device's copy of the kernel)
+    AUG_CUDA_OK(cudaFuncSetAttribute(rir_image_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)smem));
     dim3 grid(c.max_sources, B);
     rir_image_kernel<<<grid, RIR_THREADS, smem, st>>>(
         table, c.max_sources, c.rir_taps, c.frac_half_width, (double)c.fs, (double)c.sound_speed,
