@@ -64,16 +64,19 @@ def workload_label(i):
 # ------------------------------------------------------------------ algorithmic work
 def conv_work(w):
     """Nominal flops and compulsory bytes of the convolution step for one batch, per kernel.
-    Per source one forward real FFT per 4096-sample block (2.5 F log2 F, F = 8192),
-    8 flops per bin and partition for the spectral multiply-accumulate, two inverse
-    FFTs per block.  With one partition a single fused kernel does all of it
-    (bytes: inputs read once, y_s and v written once, partition spectra read once);
-    with more, block_spectra_kernel does the forward FFTs (inputs in, block spectra
-    out) and spectral_convolve_kernel the rest (block and partition spectra in,
-    y_s and v out)."""
-    F, blk = 8192, 4096
-    P = -(-int(w.cfg["rir_taps"]) // blk)
-    fft = 2.5 * F * 13
+    Per source one forward real FFT per block (2.5 F log2 F), 8 flops per bin and
+    partition for the spectral multiply, two inverse FFTs per block (one without
+    noise).  Responses of up to 4096 / 8192 taps take one partition of an 8192- /
+    16384-point transform and a single fused kernel does all of it (bytes: inputs
+    read once, y_s and v written once, response spectra read once); longer ones are
+    cut into 4096-tap partitions: block_spectra_kernel does the forward FFTs (inputs
+    in, block spectra out) and spectral_convolve_kernel the rest (block and partition
+    spectra in, y_s and v out)."""
+    taps = int(w.cfg["rir_taps"])
+    blk = 8192 if 4096 < taps <= 8192 else 4096
+    F = 2 * blk
+    P = -(-taps // blk)
+    fft = 2.5 * F * np.log2(F)
     spec = (F // 2) * 8.0
     fwd_f = fwd_b = fin_f = fin_b = 0.0
     for b in range(w.B):

@@ -33,7 +33,7 @@ int check_config(const AugConfig *c) {
 }
 
 struct Layout {
-    int n_part, n_bins, t_cap, nblk_cap;
+    int n_part, route, n_bins, t_cap, nblk_cap;
     int64_t ws_stride;
     int64_t off_xspec;
     int64_t off_tw, off_rir, off_hspec, off_ys, off_vv, off_energy, off_gain, off_melw, off_melstart,
@@ -44,6 +44,7 @@ struct Layout {
 Layout make_layout(const AugConfig &c) {
     Layout l;
     l.n_part = (c.rir_taps + aug::CONV_BLK - 1) / aug::CONV_BLK;
+    l.route = l.n_part == 1 ? aug::ROUTE_FUSED_4096 : l.n_part == 2 ? aug::ROUTE_FUSED_8192 : aug::ROUTE_STORED;
     l.n_bins = c.n_fft / 2 + 1;
     l.t_cap = aug_frame_count(c.max_samples, c.win, c.hop);
     l.ws_stride = align_up(c.max_samples, 4);
@@ -54,7 +55,7 @@ Layout make_layout(const AugConfig &c) {
     l.off_rir = take(sizeof(float) * B * S * c.rir_taps);
     l.off_hspec = take(sizeof(float2) * B * S * l.n_part * aug::CONV_N2);
     l.nblk_cap = (c.max_samples + aug::CONV_BLK - 1) / aug::CONV_BLK;
-    l.off_xspec = l.n_part > 1 ? take(sizeof(float2) * B * S * l.nblk_cap * aug::CONV_N2) : -1;
+    l.off_xspec = l.route == aug::ROUTE_STORED ? take(sizeof(float2) * B * S * l.nblk_cap * aug::CONV_N2) : -1;
     l.off_ys = take(sizeof(float) * B * l.ws_stride);
     l.off_vv = take(sizeof(float) * B * l.ws_stride);
     l.off_energy = take(sizeof(double) * 2 * B);
@@ -161,6 +162,7 @@ int aug_create(AugCtx **out, const AugConfig *cfg, void *cuda_stream) {
     }
     const Layout l = make_layout(*cfg);
     ctx->n_part = l.n_part;
+    ctx->route = l.route;
     ctx->n_bins = l.n_bins;
     ctx->t_cap = l.t_cap;
     ctx->ws_stride = l.ws_stride;

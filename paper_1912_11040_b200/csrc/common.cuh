@@ -21,6 +21,12 @@ constexpr int EV_RING = 256;
 #endif
 constexpr int HOST_CHUNKS = AUG_HOST_CHUNKS;   // pipeline depth of aug_pipeline_host
 
+// How step 2 is run, fixed by the response length at aug_create:
+//   ROUTE_FUSED_4096  rir_taps <= 4096: one partition of an 8192-point transform, one kernel
+//   ROUTE_FUSED_8192  rir_taps <= 8192: one partition of a 16384-point transform, one kernel
+//   ROUTE_STORED      longer: partitions of 4096 taps, block spectra stored once and reused
+enum Route { ROUTE_FUSED_4096 = 0, ROUTE_FUSED_8192 = 1, ROUTE_STORED = 2 };
+
 enum Reason { R_NONE = 0, R_NSRC = 1, R_ORDER = 2, R_NOISE = 3 };
 
 // Per-bin entry of the warped filterbank: the bin lies in edge interval `seg`
@@ -37,6 +43,7 @@ struct AugCtx {
     cudaStream_t stream;
     int device;
     int n_part;            // RIR partitions of CONV_BLK taps
+    int route;             // aug::Route
     int n_bins;            // n_fft/2 + 1
     int t_cap;             // frames of an utterance of max_samples
     int64_t ws_stride;     // row stride (floats) of the y_s / v workspaces
@@ -46,7 +53,7 @@ struct AugCtx {
     float2 *tw;            // [TW_N] twiddles
     float *rir;            // [max_batch][max_sources][rir_taps]
     float2 *hspec;         // [max_batch][max_sources][n_part][CONV_N2]
-    float2 *xspec;         // [max_batch][max_sources][nblk_cap][CONV_N2]; NULL when n_part == 1
+    float2 *xspec;         // [max_batch][max_sources][nblk_cap][CONV_N2]; NULL unless route == ROUTE_STORED
     int nblk_cap;          // blocks of an utterance of max_samples
     float *ys;             // [max_batch][ws_stride]
     float *vv;             // [max_batch][ws_stride]

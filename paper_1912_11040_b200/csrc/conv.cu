@@ -422,22 +422,346 @@ mix_kernel(const float *__restrict__ ys, const float *__restrict__ vv, int64_t w
     }
 }
 
+// ================================================================ 8192-sample blocks
+// Impulse responses of 4097..8192 taps fit one partition of a 16384-point real
+// transform, so a CTA can do the whole block -- forward, multiply, inverse --
+// without any stored spectra.  The 8192-point complex transform of the (even, odd)
+// pairs is run as two 4096-point transforms (pairs 0, 2, 4, ... in buffer A, pairs
+// 1, 3, 5, ... in buffer B: one 128-bit load feeds one point of each) joined by a
+// radix-2 step.  Thread t owns, for k = t + 256 q < 2048, slots k and 4096-k of
+// both buffers; from those four numbers it forms bins k, 8192-k, 4096-k and
+// 4096+k of the real signal's spectrum, multiplies them with the response's
+// bins, and folds the products back into the two half-size inputs of the inverse
+// transform -- in place, with no exchange between threads.  Spectra are stored as
+// 8192 complex numbers, bins 0 and 8192 (both real) packed into slot 0.
+constexpr int BLK2 = 2 * BLK;          // output samples per block
+constexpr int F2 = 2 * BLK2;           // real transform size
+constexpr int NB2 = F2 / 2;            // complex bins stored per spectrum
+constexpr int NQ2 = N2 / 2 / CT;       // slot pairs per thread and buffer
+
+// 2*BLK2 input samples starting at `base`: thread t gets samples
+// base + 4 (t + 256 r) + {0,1} as point r of buffer A and + {2,3} as point r of B.
+__device__ __forceinline__ void load_segment4(float2 (*va)[E], float2 (*vb)[E],
+                                              const float *__restrict__ x, bool looped, int nlen,
+                                              int base, int N, int t) {
+    if (!looped) {
+#pragma unroll
+        for (int r = 0; r < E; ++r) {
+            const int i0 = base + 4 * (t + CT * r);
+            float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (i0 >= 0) {
+                if (i0 + 3 < N) {
+                    z = __ldg(reinterpret_cast<const float4 *>(x + i0));
+                } else {
+                    if (i0 < N) z.x = x[i0];
+                    if (i0 + 1 < N) z.y = x[i0 + 1];
+                    if (i0 + 2 < N) z.z = x[i0 + 2];
+                }
+            }
+            va[0][r] = make_float2(z.x, z.y);
+            vb[0][r] = make_float2(z.z, z.w);
+        }
+        return;
+    }
+    const int first = base + 4 * t;
+    const int step = (4 * CT) % nlen;
+    int m = first >= 0 ? first % nlen : (nlen - (-first) % nlen) % nlen;
+#pragma unroll
+    for (int r = 0; r < E; ++r) {
+        const int i0 = first + 4 * CT * r;
+        float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (i0 >= 0 && i0 < N) {
+            int j = m;
+            z.x = x[j];
+            j = j + 1 == nlen ? 0 : j + 1;
+            if (i0 + 1 < N) z.y = x[j];
+            j = j + 1 == nlen ? 0 : j + 1;
+            if (i0 + 2 < N) z.z = x[j];
+            j = j + 1 == nlen ? 0 : j + 1;
+            if (i0 + 3 < N) z.w = x[j];
+        }
+        va[0][r] = make_float2(z.x, z.y);
+        vb[0][r] = make_float2(z.z, z.w);
+        m += step;
+        if (m >= nlen) m -= nlen;
+    }
+}
+
+// Both half transforms of a segment held in registers; on return A and B hold the
+// 4096-point transforms of the even and odd pairs, complete and synchronised.
+__device__ __forceinline__ void fft2x4096_from_regs(float2 (*va)[E], float2 (*vb)[E], float2 *A,
+                                                    float2 *B, int t, const float2 *__restrict__ tw) {
+    pass_from_regs<N2, E, 16, 1>(va, A, t, tw);
+    pass_from_regs<N2, E, 16, 1>(vb, B, t, tw);
+    __syncthreads();
+    pass_pair<N2, E, 16, 16, 1>(A, B, t, tw, CtaSync());
+    pass_pair<N2, E, 16, 256, 16>(A, B, t, tw, CtaSync());
+    __syncthreads();
+}
+
+__device__ __forceinline__ void fft2x4096_in_place(float2 *A, float2 *B, int t,
+                                                   const float2 *__restrict__ tw) {
+    pass_pair<N2, E, 16, 1, 0>(A, B, t, tw, CtaSync());
+    pass_pair<N2, E, 16, 16, 1>(A, B, t, tw, CtaSync());
+    pass_pair<N2, E, 16, 256, 16>(A, B, t, tw, CtaSync());
+    __syncthreads();
+}
+
+// Inverse of real_split, unnormalised (twice the value): the half-size spectrum
+// at the bin pair (k, M-k) from the real signal's bins Y[k], Y[M-k]; W = W_{2M}^k.
+__device__ __forceinline__ void real_unsplit(float2 yk, float2 ym, float2 w, float2 &zk, float2 &zm) {
+    const float2 a = make_float2(yk.x + ym.x, yk.y - ym.y);          // Yk + conj Ym
+    const float2 d = make_float2(yk.x - ym.x, yk.y + ym.y);          // Yk - conj Ym
+    const float2 e = cmul(make_float2(w.y, w.x), d);                 // i conj(W) d
+    zk = make_float2(a.x + e.x, a.y + e.y);
+    const float2 e2 = cmul(make_float2(-w.y, w.x), make_float2(d.x, -d.y));   // i W conj(d)
+    zm = make_float2(a.x + e2.x, -a.y + e2.y);
+}
+
+// The four bins a thread forms for slot k (1 <= k < 2048) from the two half
+// transforms: X[k], X[8192-k], X[4096-k], X[4096+k].
+struct Quad {
+    float2 k, nk, mk, pk;
+};
+__device__ __forceinline__ Quad quad_forward(float2 ze_k, float2 ze_m, float2 zo_k, float2 zo_m,
+                                             float2 w, float2 u) {
+    // radix-2 join: Z[k], Z[k+4096], Z[4096-k], Z[8192-k]
+    const float2 t1 = cmul(w, zo_k), t2 = cmul(cconj(w), zo_m);
+    const float2 z_k = cadd(ze_k, t1), z_pk = csub(ze_k, t1);
+    const float2 z_mk = csub(ze_m, t2), z_nk = cadd(ze_m, t2);
+    Quad x;
+    real_split(z_k, z_nk, u, x.k, x.nk);
+    real_split(z_mk, z_pk, make_float2(-u.y, -u.x), x.mk, x.pk);    // W_F^(4096-k) = -i conj(u)
+    return x;
+}
+// Products back to the inputs of the two half-size inverse transforms, real and
+// imaginary parts swapped (the forward code then computes the inverse).
+__device__ __forceinline__ void quad_inverse(const Quad &y, float2 w, float2 u, float2 &a_k,
+                                             float2 &a_m, float2 &b_k, float2 &b_m) {
+    float2 z_k, z_nk, z_mk, z_pk;
+    real_unsplit(y.k, y.nk, u, z_k, z_nk);
+    real_unsplit(y.mk, y.pk, make_float2(-u.y, -u.x), z_mk, z_pk);
+    const float2 s1 = cadd(z_k, z_pk), d1 = cmul(csub(z_k, z_pk), cconj(w));
+    const float2 s2 = cadd(z_mk, z_nk), d2 = cmul(csub(z_nk, z_mk), w);   // -(Z[4096-k]-Z[8192-k]) w
+    a_k = make_float2(s1.y, s1.x);
+    b_k = make_float2(d1.y, d1.x);
+    a_m = make_float2(s2.y, s2.x);
+    b_m = make_float2(d2.y, d2.x);
+}
+
+// Slots 0 and 2048 of both buffers (thread 0): bins 0, 8192 (packed), 4096, 2048, 6144.
+struct Edge {
+    float2 dc;       // (X[0], X[8192]), both real
+    float2 mid;      // X[4096]
+    float2 q1, q3;   // X[2048], X[6144]
+};
+__device__ __forceinline__ Edge edge_forward(float2 ze0, float2 zo0, float2 zeh, float2 zoh, float2 uh) {
+    Edge x;
+    const float2 z0 = cadd(ze0, zo0), z4 = csub(ze0, zo0);
+    x.dc = make_float2(z0.x + z0.y, z0.x - z0.y);
+    x.mid = cconj(z4);
+    const float2 th = cmul_mi(zoh);                                 // W_8192^2048 = -i
+    real_split(cadd(zeh, th), csub(zeh, th), uh, x.q1, x.q3);
+    return x;
+}
+__device__ __forceinline__ void edge_inverse(const Edge &y, float2 uh, float2 &a0, float2 &b0,
+                                             float2 &ah, float2 &bh) {
+    const float2 z0 = make_float2(y.dc.x + y.dc.y, y.dc.x - y.dc.y);
+    const float2 z4 = make_float2(2.f * y.mid.x, -2.f * y.mid.y);
+    const float2 s0 = cadd(z0, z4), d0 = csub(z0, z4);
+    float2 z2, z6;
+    real_unsplit(y.q1, y.q3, uh, z2, z6);
+    const float2 sh = cadd(z2, z6), dd = csub(z2, z6);
+    const float2 dh = make_float2(-dd.y, dd.x);                     // times conj(-i) = i
+    a0 = make_float2(s0.y, s0.x);
+    b0 = make_float2(d0.y, d0.x);
+    ah = make_float2(sh.y, sh.x);
+    bh = make_float2(dh.y, dh.x);
+}
+
+// Spectrum of one 16384-sample segment of each impulse response (taps beyond L and
+// the whole second half are zero), scaled by the noise weight and 1/F.
+__global__ void __launch_bounds__(CT)
+rir_spectra2_kernel(const float *__restrict__ rir, const AugUttParams *__restrict__ table, int S_max,
+                    int L, const float2 *__restrict__ tw, float2 *__restrict__ hspec) {
+    extern __shared__ __align__(16) float2 sm[];
+    float2 *A = sm, *Bf = sm + SM_POINTS;
+    const int s = blockIdx.x, utt = blockIdx.y, t = threadIdx.x;
+    const AugUttParams &row = table[utt];
+    if (row.n_src < 1 || row.n_src > S_max || s >= row.n_src) return;
+    const float scale = (s == 0 ? 1.f : row.noise_weight[s - 1]) / (float)F2;
+    const float *h = rir + ((int64_t)utt * S_max + s) * L;
+    float2 *out = hspec + ((int64_t)utt * S_max + s) * NB2;
+    {
+        float2 va[1][E], vb[1][E];
+#pragma unroll
+        for (int r = 0; r < E; ++r) {
+            const int i0 = 4 * (t + CT * r);
+            float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (i0 < BLK2) {
+                if (i0 < L) z.x = h[i0];
+                if (i0 + 1 < L) z.y = h[i0 + 1];
+                if (i0 + 2 < L) z.z = h[i0 + 2];
+                if (i0 + 3 < L) z.w = h[i0 + 3];
+            }
+            va[0][r] = make_float2(z.x, z.y);
+            vb[0][r] = make_float2(z.z, z.w);
+        }
+        fft2x4096_from_regs(va, vb, A, Bf, t, tw);
+    }
+#pragma unroll
+    for (int q = 0; q < NQ2; ++q) {
+        const int k = t + CT * q;
+        if (k == 0) {
+            const Edge x = edge_forward(A[pad0(0)], Bf[pad0(0)], A[pad0(N2 / 2)], Bf[pad0(N2 / 2)],
+                                        __ldg(&tw[tw_index(F2, N2 / 2)]));
+            out[0] = make_float2(x.dc.x * scale, x.dc.y * scale);
+            out[N2] = make_float2(x.mid.x * scale, x.mid.y * scale);
+            out[N2 / 2] = make_float2(x.q1.x * scale, x.q1.y * scale);
+            out[N2 + N2 / 2] = make_float2(x.q3.x * scale, x.q3.y * scale);
+        } else {
+            const Quad x = quad_forward(A[pad0(k)], A[pad0(N2 - k)], Bf[pad0(k)], Bf[pad0(N2 - k)],
+                                        __ldg(&tw[tw_index(NB2, k)]), __ldg(&tw[tw_index(F2, k)]));
+            out[k] = make_float2(x.k.x * scale, x.k.y * scale);
+            out[NB2 - k] = make_float2(x.nk.x * scale, x.nk.y * scale);
+            out[N2 - k] = make_float2(x.mk.x * scale, x.mk.y * scale);
+            out[N2 + k] = make_float2(x.pk.x * scale, x.pk.y * scale);
+        }
+    }
+}
+
+__global__ void __launch_bounds__(CT, CONV_MINB)
+convolve_fused2_kernel(const float *__restrict__ speech, int64_t stride,
+                       const int *__restrict__ lengths, const float *__restrict__ bank,
+                       int64_t bank_len, const AugUttParams *__restrict__ table, int S_max,
+                       const float2 *__restrict__ hspec, const float2 *__restrict__ tw,
+                       float *__restrict__ ys, float *__restrict__ vv, int64_t ws_stride,
+                       double *__restrict__ energy, int *status, int n_cap) {
+    extern __shared__ __align__(16) float2 sm[];
+    float2 *A = sm, *Bf = sm + SM_POINTS;
+    __shared__ float red[CT / 32];
+    const int b = blockIdx.x, utt = blockIdx.y, t = threadIdx.x;
+    const int N = min(max(lengths[utt], 0), n_cap);
+    if ((int64_t)b * BLK2 >= N) return;
+    const AugUttParams &row = table[utt];
+    int n_src = row.n_src;
+    if (n_src < 1 || n_src > S_max) n_src = 0;   // rejected row: silence (reported by step 1)
+    const int n_left = N - b * BLK2;
+
+    // Noise sources are summed in the time domain (v is read back and added to for
+    // every source after the first); the energy is taken when the last one lands.
+    int last_noise = 0;
+    for (int s = 1; s < n_src; ++s) {
+        const float *x;
+        int nlen;
+        if (source_of(row, s, nullptr, bank, bank_len, x, nlen)) last_noise = s;
+        else if (t == 0 && b == 0 && atomicCAS(&status[0], -1, utt) == -1) status[1] = aug::R_NOISE;
+    }
+    bool v_written = false;
+    for (int s = 0; s < n_src; ++s) {
+        const float *x;
+        int nlen;
+        if (!source_of(row, s, speech + (int64_t)utt * stride, bank, bank_len, x, nlen)) continue;
+        {
+            float2 va[1][E], vb[1][E];
+            load_segment4(va, vb, x, s != 0, nlen, (b - 1) * BLK2, N, t);
+            fft2x4096_from_regs(va, vb, A, Bf, t, tw);
+        }
+        const float2 *H = hspec + ((int64_t)utt * S_max + s) * NB2;
+#pragma unroll 2
+        for (int q = 0; q < NQ2; ++q) {
+            const int k = t + CT * q;
+            if (k == 0) {
+                const float2 uh = __ldg(&tw[tw_index(F2, N2 / 2)]);
+                Edge x4 = edge_forward(A[pad0(0)], Bf[pad0(0)], A[pad0(N2 / 2)], Bf[pad0(N2 / 2)], uh);
+                const float2 h0 = __ldg(&H[0]);
+                x4.dc = make_float2(x4.dc.x * h0.x, x4.dc.y * h0.y);
+                x4.mid = cmul(x4.mid, __ldg(&H[N2]));
+                x4.q1 = cmul(x4.q1, __ldg(&H[N2 / 2]));
+                x4.q3 = cmul(x4.q3, __ldg(&H[N2 + N2 / 2]));
+                edge_inverse(x4, uh, A[pad0(0)], Bf[pad0(0)], A[pad0(N2 / 2)], Bf[pad0(N2 / 2)]);
+            } else {
+                const float2 w = __ldg(&tw[tw_index(NB2, k)]), u = __ldg(&tw[tw_index(F2, k)]);
+                Quad x4 = quad_forward(A[pad0(k)], A[pad0(N2 - k)], Bf[pad0(k)], Bf[pad0(N2 - k)], w, u);
+                x4.k = cmul(x4.k, __ldg(&H[k]));
+                x4.nk = cmul(x4.nk, __ldg(&H[NB2 - k]));
+                x4.mk = cmul(x4.mk, __ldg(&H[N2 - k]));
+                x4.pk = cmul(x4.pk, __ldg(&H[N2 + k]));
+                quad_inverse(x4, w, u, A[pad0(k)], A[pad0(N2 - k)], Bf[pad0(k)], Bf[pad0(N2 - k)]);
+            }
+        }
+        __syncthreads();
+        fft2x4096_in_place(A, Bf, t, tw);
+
+        // Outputs 8192..16383 of the segment are this block: pair 4096 + 2 j is point
+        // 2048 + j of A (samples 4j, 4j+1), pair 4096 + 2 j + 1 the same point of B.
+        const bool is_speech = s == 0;
+        const bool add = !is_speech && v_written;
+        const bool want_energy = is_speech || s == last_noise;
+        float *dst = (is_speech ? ys : vv) + (int64_t)utt * ws_stride + (int64_t)b * BLK2;
+        float e2sum = 0.f;
+#pragma unroll
+        for (int r = 0; r < BLK2 / 4 / CT; ++r) {
+            const int j = t + CT * r;
+            const float2 za = A[pad0(N2 / 2 + j)], zb = Bf[pad0(N2 / 2 + j)];
+            float4 y = make_float4(za.y, za.x, zb.y, zb.x);
+            const int i = 4 * j;
+            if (i + 3 < n_left) {
+                float4 *p = reinterpret_cast<float4 *>(dst + i);
+                if (add) {
+                    const float4 o = *p;
+                    y = make_float4(y.x + o.x, y.y + o.y, y.z + o.z, y.w + o.w);
+                }
+                *p = y;
+                e2sum += y.x * y.x + y.y * y.y + y.z * y.z + y.w * y.w;
+            } else {
+                const float yy[3] = {y.x, y.y, y.z};
+                for (int c = 0; c < 3 && i + c < n_left; ++c) {
+                    const float val = add ? yy[c] + dst[i + c] : yy[c];
+                    dst[i + c] = val;
+                    e2sum += val * val;
+                }
+            }
+        }
+        if (want_energy) {
+            const float tot = block_sum(e2sum, red, t);
+            if (t == 0) atomicAdd(&energy[2 * utt + (is_speech ? 0 : 1)], (double)tot);
+        }
+        if (!is_speech) v_written = true;
+        __syncthreads();   // the buffers are refilled by the next source
+    }
+    if (!v_written) {
+        // no (usable) noise: v is defined as silence
+        float *dst = vv + (int64_t)utt * ws_stride + (int64_t)b * BLK2;
+        for (int i = t; i < BLK2 && i < n_left; i += CT) dst[i] = 0.f;
+    }
+}
+
 constexpr size_t FFT_SMEM = sizeof(float2) * SM_POINTS;
+constexpr size_t FFT2_SMEM = 2 * FFT_SMEM;
 
 }  // namespace
 
 int launch_rir_spectra(AugCtx *ctx, const float *rir, const AugUttParams *table, int B,
                        cudaStream_t st) {
     const AugConfig &c = ctx->cfg;
-    dim3 grid(ctx->n_part, c.max_sources, B);
-    rir_spectra_kernel<<<grid, CT, FFT_SMEM, st>>>(rir, table, c.max_sources, c.rir_taps,
-                                                            ctx->n_part, ctx->tw, ctx->hspec);
+    if (ctx->route == aug::ROUTE_FUSED_8192) {
+        AUG_CUDA_OK(cudaFuncSetAttribute(rir_spectra2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)FFT2_SMEM));
+        dim3 grid(c.max_sources, B);
+        rir_spectra2_kernel<<<grid, CT, FFT2_SMEM, st>>>(rir, table, c.max_sources, c.rir_taps, ctx->tw,
+                                                         ctx->hspec);
+    } else {
+        dim3 grid(ctx->n_part, c.max_sources, B);
+        rir_spectra_kernel<<<grid, CT, FFT_SMEM, st>>>(rir, table, c.max_sources, c.rir_taps,
+                                                       ctx->n_part, ctx->tw, ctx->hspec);
+    }
     AUG_CUDA_OK(cudaGetLastError());
     ctx->launches++;
     return AUG_OK;
 }
 
-static bool stored_route(const AugCtx *ctx) { return ctx->n_part > 1 && ctx->xspec != nullptr; }
+static bool stored_route(const AugCtx *ctx) { return ctx->route == aug::ROUTE_STORED; }
 
 int launch_convolve_prepare(AugCtx *ctx, const float *speech, int64_t stride, const int *lengths,
                             const float *bank, int64_t bank_len, const AugUttParams *table, int B,
@@ -463,7 +787,14 @@ int launch_convolve_finish(AugCtx *ctx, const float *speech, int64_t stride, con
     if (max_len <= 0) return AUG_OK;
     const int nblk = (max_len + BLK - 1) / BLK;
     dim3 grid(nblk, B);
-    if (!stored_route(ctx)) {
+    if (ctx->route == aug::ROUTE_FUSED_8192) {
+        AUG_CUDA_OK(cudaFuncSetAttribute(convolve_fused2_kernel,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FFT2_SMEM));
+        dim3 grid2((max_len + BLK2 - 1) / BLK2, B);
+        convolve_fused2_kernel<<<grid2, CT, FFT2_SMEM, ctx->stream>>>(
+            speech, stride, lengths, bank, bank_len, table, c.max_sources, ctx->hspec, ctx->tw,
+            ctx->ys, ctx->vv, ctx->ws_stride, ctx->energy, ctx->status, max_len);
+    } else if (!stored_route(ctx)) {
         convolve_fused_kernel<<<grid, CT, FFT_SMEM, ctx->stream>>>(
             speech, stride, lengths, bank, bank_len, table, c.max_sources, ctx->n_part, ctx->hspec,
             ctx->tw, ctx->ys, ctx->vv, ctx->ws_stride, ctx->energy, ctx->status, max_len);

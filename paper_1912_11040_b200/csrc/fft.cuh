@@ -156,24 +156,49 @@ __device__ __forceinline__ void pass_from_regs(float2 (*v)[R], float2 *s, int t,
     }
 }
 
-// A full pass: gather from `s` (laid out by the pass whose NS was NS_PREV; 0 when
-// the caller wrote the input with shift 0), barrier, transform, scatter, barrier.
-template <int N, int E, int R, int NS, int NS_PREV, typename Sync>
-__device__ __forceinline__ void pass(float2 *s, int t, const float2 *__restrict__ tw, Sync sync) {
+// Gather the inputs of this thread's butterflies from `s`, laid out by the pass
+// whose NS was NS_PREV (0 when the caller wrote the input with shift 0).
+template <int N, int E, int R, int NS_PREV>
+__device__ __forceinline__ void gather(float2 (*v)[R], const float2 *s, int t) {
     constexpr int T = N / E;
     constexpr int NB = E / R;
     constexpr int PS_IN = out_shift(NS_PREV);
-    float2 v[NB][R];
+    static_assert((N / R) % 16 == 0, "gather stride must keep the row offset constant");
 #pragma unroll
     for (int b = 0; b < NB; ++b) {
-        static_assert((N / R) % 16 == 0, "gather stride must keep the row offset constant");
         const int base = padi<PS_IN>(t + b * T);
 #pragma unroll
         for (int r = 0; r < R; ++r) v[b][r] = s[base + padi<PS_IN>(r * (N / R))];
     }
+}
+
+// A full pass: gather, barrier, transform, scatter, barrier.
+template <int N, int E, int R, int NS, int NS_PREV, typename Sync>
+__device__ __forceinline__ void pass(float2 *s, int t, const float2 *__restrict__ tw, Sync sync) {
+    constexpr int NB = E / R;
+    float2 v[NB][R];
+    gather<N, E, R, NS_PREV>(v, s, t);
     sync();
     pass_from_regs<N, E, R, NS>(v, s, t, tw);
     sync();
+}
+
+// The same pass on two independent transforms in buffers `a` and `b`: the barrier
+// that lets `a` be overwritten also publishes the previous writes to `b`, so the
+// pair costs two barriers, not four.  On entry both buffers must be complete and
+// visible; on exit `a` is complete and visible, `b` is written but not yet
+// synchronised (the next pass_pair, or one barrier, finishes it).
+template <int N, int E, int R, int NS, int NS_PREV, typename Sync>
+__device__ __forceinline__ void pass_pair(float2 *a, float2 *b, int t, const float2 *__restrict__ tw,
+                                          Sync sync) {
+    constexpr int NB = E / R;
+    float2 v[NB][R];
+    gather<N, E, R, NS_PREV>(v, a, t);
+    sync();
+    pass_from_regs<N, E, R, NS>(v, a, t, tw);
+    gather<N, E, R, NS_PREV>(v, b, t);
+    sync();
+    pass_from_regs<N, E, R, NS>(v, b, t, tw);
 }
 
 struct CtaSync {
