@@ -44,7 +44,8 @@ struct Layout {
 Layout make_layout(const AugConfig &c) {
     Layout l;
     l.n_part = (c.rir_taps + aug::CONV_BLK - 1) / aug::CONV_BLK;
-    l.route = l.n_part == 1 ? aug::ROUTE_FUSED_4096 : l.n_part == 2 ? aug::ROUTE_FUSED_8192 : aug::ROUTE_STORED;
+    l.route = c.rir_taps <= aug::FUSED16K_MIN_TAPS ? aug::ROUTE_FUSED_4096
+              : l.n_part <= 2 ? aug::ROUTE_FUSED_8192 : aug::ROUTE_STORED;
     l.n_bins = c.n_fft / 2 + 1;
     l.t_cap = aug_frame_count(c.max_samples, c.win, c.hop);
     l.ws_stride = align_up(c.max_samples, 4);
@@ -53,7 +54,7 @@ Layout make_layout(const AugConfig &c) {
     auto take = [&](int64_t bytes) { int64_t r = o; o = align_up(o + bytes, 256); return r; };
     l.off_tw = take(sizeof(float2) * augfft::TW_N);
     l.off_rir = take(sizeof(float) * B * S * c.rir_taps);
-    l.off_hspec = take(sizeof(float2) * B * S * l.n_part * aug::CONV_N2);
+    l.off_hspec = take(sizeof(float2) * B * S * (l.route == aug::ROUTE_FUSED_8192 ? 2 : l.n_part) * aug::CONV_N2);
     l.nblk_cap = (c.max_samples + aug::CONV_BLK - 1) / aug::CONV_BLK;
     l.off_xspec = l.route == aug::ROUTE_STORED ? take(sizeof(float2) * B * S * l.nblk_cap * aug::CONV_N2) : -1;
     l.off_ys = take(sizeof(float) * B * l.ws_stride);

@@ -636,17 +636,18 @@ convolve_fused2_kernel(const float *__restrict__ speech, int64_t stride,
                        int64_t bank_len, const AugUttParams *__restrict__ table, int S_max,
                        const float2 *__restrict__ hspec, const float2 *__restrict__ tw,
                        float *__restrict__ ys, float *__restrict__ vv, int64_t ws_stride,
-                       double *__restrict__ energy, int *status, int n_cap) {
+                       double *__restrict__ energy, int *status, int n_cap, int ob) {
     extern __shared__ __align__(16) float2 sm[];
     float2 *A = sm, *Bf = sm + SM_POINTS;
     __shared__ float red[CT / 32];
     const int b = blockIdx.x, utt = blockIdx.y, t = threadIdx.x;
     const int N = min(max(lengths[utt], 0), n_cap);
-    if ((int64_t)b * BLK2 >= N) return;
+    if ((int64_t)b * ob >= N) return;
     const AugUttParams &row = table[utt];
     int n_src = row.n_src;
     if (n_src < 1 || n_src > S_max) n_src = 0;   // rejected row: silence (reported by step 1)
-    const int n_left = N - b * BLK2;
+    const int n_left = min(N - b * ob, ob);
+    const int m0 = (F2 - ob) / 4;            // first point of A and B that belongs to this block
 
     // Noise sources are summed in the time domain (v is read back and added to for
     // every source after the first); the energy is taken when the last one lands.
@@ -664,7 +665,7 @@ convolve_fused2_kernel(const float *__restrict__ speech, int64_t stride,
         if (!source_of(row, s, speech + (int64_t)utt * stride, bank, bank_len, x, nlen)) continue;
         {
             float2 va[1][E], vb[1][E];
-            load_segment4(va, vb, x, s != 0, nlen, (b - 1) * BLK2, N, t);
+            load_segment4(va, vb, x, s != 0, nlen, (b + 1) * ob - F2, N, t);
             fft2x4096_from_regs(va, vb, A, Bf, t, tw);
         }
         const float2 *H = hspec + ((int64_t)utt * S_max + s) * NB2;
@@ -693,17 +694,16 @@ convolve_fused2_kernel(const float *__restrict__ speech, int64_t stride,
         __syncthreads();
         fft2x4096_in_place(A, Bf, t, tw);
 
-        // Outputs 8192..16383 of the segment are this block: pair 4096 + 2 j is point
-        // 2048 + j of A (samples 4j, 4j+1), pair 4096 + 2 j + 1 the same point of B.
+        // The last `ob` outputs of the segment are this block: samples 4m, 4m+1 of the
+        // segment are point m of A, samples 4m+2, 4m+3 point m of B.
         const bool is_speech = s == 0;
         const bool add = !is_speech && v_written;
         const bool want_energy = is_speech || s == last_noise;
-        float *dst = (is_speech ? ys : vv) + (int64_t)utt * ws_stride + (int64_t)b * BLK2;
+        float *dst = (is_speech ? ys : vv) + (int64_t)utt * ws_stride + (int64_t)b * ob;
         float e2sum = 0.f;
-#pragma unroll
-        for (int r = 0; r < BLK2 / 4 / CT; ++r) {
-            const int j = t + CT * r;
-            const float2 za = A[pad0(N2 / 2 + j)], zb = Bf[pad0(N2 / 2 + j)];
+#pragma unroll 4
+        for (int j = t; m0 + j < N2; j += CT) {
+            const float2 za = A[pad0(m0 + j)], zb = Bf[pad0(m0 + j)];
             float4 y = make_float4(za.y, za.x, zb.y, zb.x);
             const int i = 4 * j;
             if (i + 3 < n_left) {
@@ -732,8 +732,8 @@ convolve_fused2_kernel(const float *__restrict__ speech, int64_t stride,
     }
     if (!v_written) {
         // no (usable) noise: v is defined as silence
-        float *dst = vv + (int64_t)utt * ws_stride + (int64_t)b * BLK2;
-        for (int i = t; i < BLK2 && i < n_left; i += CT) dst[i] = 0.f;
+        float *dst = vv + (int64_t)utt * ws_stride + (int64_t)b * ob;
+        for (int i = t; i < n_left; i += CT) dst[i] = 0.f;
     }
 }
 
@@ -790,10 +790,12 @@ int launch_convolve_finish(AugCtx *ctx, const float *speech, int64_t stride, con
     if (ctx->route == aug::ROUTE_FUSED_8192) {
         AUG_CUDA_OK(cudaFuncSetAttribute(convolve_fused2_kernel,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FFT2_SMEM));
-        dim3 grid2((max_len + BLK2 - 1) / BLK2, B);
+        // every block yields the F2 - (taps - 1) outputs that see no wrap-around, cut to a multiple of 4
+        const int ob = (F2 - c.rir_taps + 1) & ~3;
+        dim3 grid2((max_len + ob - 1) / ob, B);
         convolve_fused2_kernel<<<grid2, CT, FFT2_SMEM, ctx->stream>>>(
             speech, stride, lengths, bank, bank_len, table, c.max_sources, ctx->hspec, ctx->tw,
-            ctx->ys, ctx->vv, ctx->ws_stride, ctx->energy, ctx->status, max_len);
+            ctx->ys, ctx->vv, ctx->ws_stride, ctx->energy, ctx->status, max_len, ob);
     } else if (!stored_route(ctx)) {
         convolve_fused_kernel<<<grid, CT, FFT_SMEM, ctx->stream>>>(
             speech, stride, lengths, bank, bank_len, table, c.max_sources, ctx->n_part, ctx->hspec,

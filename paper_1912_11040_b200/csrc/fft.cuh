@@ -117,17 +117,21 @@ __device__ __forceinline__ void twiddle(float2 *v, float2 w1) {
 }
 
 // Shared-memory index padding.  Complex points are 8 bytes, 16 of them span the 32
-// banks; element i lives at i + ((i >> 4) << PS), i.e. every row of 16 points is
-// shifted by 1 (PS = 0) or 2 (PS = 1) slots per row.  Row-constant shifts keep the
-// unit-stride gathers conflict-free; the shift is chosen per pass so that its
-// scatter is conflict-free too: stride-R scatters (NS = 1) want 1 per row, the
-// NS = 8 scatter (rows 4 apart within a half-warp) wants 2 per row.
+// banks.  Between passes element i lives at i + ((i >> 4) << PS), i.e. every row of
+// 16 points is shifted by 1 (PS = 0) or 2 (PS = 1) slots per row.  Row-constant
+// shifts keep the unit-stride gathers conflict-free; the shift is chosen per pass
+// so that its scatter is conflict-free too: stride-R scatters (NS = 1) and the
+// NS = 16 scatter want 1 per row, the NS = 8 scatter (rows 4 apart within a
+// half-warp) wants 2 per row.  The last pass of a transform (NS >= 64 here) writes
+// consecutive slots from consecutive threads and so do callers that fill a buffer
+// themselves (NS = 0): those layouts are left unpadded (PS = -1), which also keeps
+// mirrored reads (slot N-k next to slot k) free of conflicts.
 template <int PS>
-__device__ __forceinline__ int padi(int i) { return i + ((i >> 4) << PS); }
+__device__ __forceinline__ int padi(int i) { return PS < 0 ? i : i + ((i >> 4) << (PS < 0 ? 0 : PS)); }
 __host__ __device__ constexpr int padded_points(int n) { return n + n / 8; }
-__host__ __device__ constexpr int out_shift(int NS) { return NS == 8 ? 1 : 0; }
-// Final-pass outputs (NS >= 64) and caller-written inputs use shift 0.
-__device__ __forceinline__ int pad0(int i) { return padi<0>(i); }
+__host__ __device__ constexpr int out_shift(int NS) { return NS == 8 ? 1 : (NS == 1 || NS == 16) ? 0 : -1; }
+// Index of point i in a finished transform or in a caller-written input: unpadded.
+__device__ __forceinline__ int pad0(int i) { return i; }
 
 // One pass over registers already holding the inputs of this thread's butterflies:
 //   v[b][r] = data[(t + b T) + r N/R],  T = N/E threads, b < E/R.
@@ -139,6 +143,7 @@ __device__ __forceinline__ void pass_from_regs(float2 (*v)[R], float2 *s, int t,
     constexpr int T = N / E;
     constexpr int NB = E / R;
     constexpr int PS = out_shift(NS);
+    static_assert(PS >= 0 || NS * R == N, "only the last pass may write the unpadded layout");
 #pragma unroll
     for (int b = 0; b < NB; ++b) {
         const int j = t + b * T;
