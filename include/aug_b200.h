@@ -94,7 +94,10 @@ typedef struct {
     float alpha;                   /* VTLP warp factor of Eq. 1, in (0,2); 1 = no warp */
     float src_pos[AUG_S_MAX][3];   /* [0] = speech source, [1..] = noise sources */
     int64_t noise_offset[AUG_S_MAX - 1]; /* start of this source's stretch of the noise bank */
-    int32_t noise_len[AUG_S_MAX - 1];    /* its length; it repeats end to end over the utterance */
+    int32_t noise_len[AUG_S_MAX - 1];    /* its length; it repeats end to end over the utterance.
+                                            Any offset and length work; stretches whose offset and
+                                            length are multiples of 4 samples are read with 128-bit
+                                            loads and convolve faster */
     float noise_weight[AUG_S_MAX - 1];   /* relative level of this source in the noise sum */
 } AugUttParams;
 
@@ -142,7 +145,9 @@ typedef struct {
 /* Draw B rows on the host from `seed` (counter-based SplitMix64: row b depends only
  * on seed and b).  Each noise source gets a stretch of the bank of length between
  * half the utterance and the whole utterance (clamped to [min_noise_len, bank_len])
- * at a uniform offset, weight 1.  Rows always pass aug_validate_params for a
+ * at a uniform offset, weight 1; offset and length are rounded down to multiples of 4
+ * samples (lengths of at least 4) so that the stretches can be read with 128-bit loads.
+ * Rows always pass aug_validate_params for a
  * configuration with max_order >= order and max_sources > n_noise_hi.
  * Returns AUG_EINVAL for null pointers or inconsistent ranges. */
 int aug_sample_params(uint64_t seed, const AugDist *dist_host, int B, const int *lengths_host,

@@ -31,6 +31,9 @@ constexpr int CT = 256;               // threads per CTA
 constexpr int E = N2 / CT;            // 16 points per thread: three radix-16 passes
 constexpr int NQ = N2 / 2 / CT;       // 8 bin pairs per thread
 constexpr int SM_POINTS = padded_points(N2);
+#ifndef CONV_RUN
+#define CONV_RUN 1                   // consecutive 16384-point blocks one CTA works through
+#endif
 #ifndef CONV_MINB
 #define CONV_MINB 3                  // CTAs per SM the register budget is set for
 #endif
@@ -466,24 +469,72 @@ __device__ __forceinline__ void load_segment4(float2 (*va)[E], float2 (*vb)[E],
     const int first = base + 4 * t;
     const int step = (4 * CT) % nlen;
     int m = first >= 0 ? first % nlen : (nlen - (-first) % nlen) % nlen;
+    if ((nlen & 3) == 0 && (reinterpret_cast<uintptr_t>(x) & 15) == 0) {
+        // A stretch that starts on a 16-byte boundary and whose length is a multiple
+        // of four samples never wraps inside a group of four: one 128-bit load each.
+#pragma unroll
+        for (int r = 0; r < E; ++r) {
+            const int i0 = first + 4 * CT * r;
+            float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (i0 >= 0 && i0 < N) {
+                z = __ldg(reinterpret_cast<const float4 *>(x + m));
+                if (i0 + 3 >= N) {
+                    z.w = 0.f;
+                    if (i0 + 2 >= N) z.z = 0.f;
+                    if (i0 + 1 >= N) z.y = 0.f;
+                }
+            }
+            va[0][r] = make_float2(z.x, z.y);
+            vb[0][r] = make_float2(z.z, z.w);
+            m += step;
+            if (m >= nlen) m -= nlen;
+        }
+        return;
+    }
 #pragma unroll
     for (int r = 0; r < E; ++r) {
         const int i0 = first + 4 * CT * r;
         float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
         if (i0 >= 0 && i0 < N) {
-            int j = m;
-            z.x = x[j];
-            j = j + 1 == nlen ? 0 : j + 1;
-            if (i0 + 1 < N) z.y = x[j];
-            j = j + 1 == nlen ? 0 : j + 1;
-            if (i0 + 2 < N) z.z = x[j];
-            j = j + 1 == nlen ? 0 : j + 1;
-            if (i0 + 3 < N) z.w = x[j];
+            if (m + 3 < nlen && i0 + 3 < N) {
+                z = make_float4(x[m], x[m + 1], x[m + 2], x[m + 3]);
+            } else {
+                int j = m;
+                z.x = x[j];
+                j = j + 1 == nlen ? 0 : j + 1;
+                if (i0 + 1 < N) z.y = x[j];
+                j = j + 1 == nlen ? 0 : j + 1;
+                if (i0 + 2 < N) z.z = x[j];
+                j = j + 1 == nlen ? 0 : j + 1;
+                if (i0 + 3 < N) z.w = x[j];
+            }
         }
         va[0][r] = make_float2(z.x, z.y);
         vb[0][r] = make_float2(z.z, z.w);
         m += step;
         if (m >= nlen) m -= nlen;
+    }
+}
+
+// Passes two and three of both half transforms, shared by the forward and the
+// inverse direction (a real call: the kernel's instruction footprint matters).
+// On entry A is complete and visible and B at most one barrier away from it.
+__device__ __noinline__ void fft2x4096_tail(float2 *A, float2 *B, int t, const float2 *__restrict__ tw) {
+    pass_pair<N2, E, 16, 16, 1>(A, B, t, tw, CtaSync());
+    pass_pair<N2, E, 16, 256, 16>(A, B, t, tw, CtaSync());
+    __syncthreads();
+}
+
+// Ask for samples [start, start + count) of a source, cut to [0, N), to be brought
+// into L2: one 128-byte line per thread and step.  A looped source maps the sample
+// index into its stretch.
+__device__ __forceinline__ void prefetch_l2(const float *x, bool looped, int nlen, int start, int count,
+                                            int N, int t) {
+    const int end = min(start + count, N);
+    for (int i = start + 32 * t; i < end; i += 32 * CT) {
+        if (i < 0) continue;
+        const float *p = x + (looped ? i % nlen : i);
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
     }
 }
 
@@ -494,17 +545,13 @@ __device__ __forceinline__ void fft2x4096_from_regs(float2 (*va)[E], float2 (*vb
     pass_from_regs<N2, E, 16, 1>(va, A, t, tw);
     pass_from_regs<N2, E, 16, 1>(vb, B, t, tw);
     __syncthreads();
-    pass_pair<N2, E, 16, 16, 1>(A, B, t, tw, CtaSync());
-    pass_pair<N2, E, 16, 256, 16>(A, B, t, tw, CtaSync());
-    __syncthreads();
+    fft2x4096_tail(A, B, t, tw);
 }
 
 __device__ __forceinline__ void fft2x4096_in_place(float2 *A, float2 *B, int t,
                                                    const float2 *__restrict__ tw) {
     pass_pair<N2, E, 16, 1, 0>(A, B, t, tw, CtaSync());
-    pass_pair<N2, E, 16, 16, 1>(A, B, t, tw, CtaSync());
-    pass_pair<N2, E, 16, 256, 16>(A, B, t, tw, CtaSync());
-    __syncthreads();
+    fft2x4096_tail(A, B, t, tw);
 }
 
 // Inverse of real_split, unnormalised (twice the value): the half-size spectrum
@@ -640,14 +687,13 @@ convolve_fused2_kernel(const float *__restrict__ speech, int64_t stride,
     extern __shared__ __align__(16) float2 sm[];
     float2 *A = sm, *Bf = sm + SM_POINTS;
     __shared__ float red[CT / 32];
-    const int b = blockIdx.x, utt = blockIdx.y, t = threadIdx.x;
+    const int b_first = blockIdx.x * CONV_RUN, utt = blockIdx.y, t = threadIdx.x;
     const int N = min(max(lengths[utt], 0), n_cap);
-    if ((int64_t)b * ob >= N) return;
+    if ((int64_t)b_first * ob >= N) return;
     const AugUttParams &row = table[utt];
     int n_src = row.n_src;
     if (n_src < 1 || n_src > S_max) n_src = 0;   // rejected row: silence (reported by step 1)
-    const int n_left = min(N - b * ob, ob);
-    const int m0 = (F2 - ob) / 4;            // first point of A and B that belongs to this block
+    const int m0 = (F2 - ob) / 4;            // first point of A and B that belongs to a block
 
     // Noise sources are summed in the time domain (v is read back and added to for
     // every source after the first); the energy is taken when the last one lands.
@@ -656,8 +702,13 @@ convolve_fused2_kernel(const float *__restrict__ speech, int64_t stride,
         const float *x;
         int nlen;
         if (source_of(row, s, nullptr, bank, bank_len, x, nlen)) last_noise = s;
-        else if (t == 0 && b == 0 && atomicCAS(&status[0], -1, utt) == -1) status[1] = aug::R_NOISE;
+        else if (t == 0 && b_first == 0 && atomicCAS(&status[0], -1, utt) == -1) status[1] = aug::R_NOISE;
     }
+    // A CTA works through CONV_RUN consecutive blocks: while it loads the segment of
+    // block b it asks for the new samples of block b + 1 to be brought into L2.
+    for (int b = b_first; b < b_first + CONV_RUN && (int64_t)b * ob < N; ++b) {
+    const int n_left = min(N - b * ob, ob);
+    const bool more = b + 1 < b_first + CONV_RUN;
     bool v_written = false;
     for (int s = 0; s < n_src; ++s) {
         const float *x;
@@ -666,6 +717,7 @@ convolve_fused2_kernel(const float *__restrict__ speech, int64_t stride,
         {
             float2 va[1][E], vb[1][E];
             load_segment4(va, vb, x, s != 0, nlen, (b + 1) * ob - F2, N, t);
+            if (more) prefetch_l2(x, s != 0, nlen, (b + 1) * ob, ob, N, t);
             fft2x4096_from_regs(va, vb, A, Bf, t, tw);
         }
         const float2 *H = hspec + ((int64_t)utt * S_max + s) * NB2;
@@ -730,11 +782,17 @@ convolve_fused2_kernel(const float *__restrict__ speech, int64_t stride,
         if (!is_speech) v_written = true;
         __syncthreads();   // the buffers are refilled by the next source
     }
+    if (n_src == 0) {
+        // rejected row: y_s is silence too
+        float *dst = ys + (int64_t)utt * ws_stride + (int64_t)b * ob;
+        for (int i = t; i < n_left; i += CT) dst[i] = 0.f;
+    }
     if (!v_written) {
         // no (usable) noise: v is defined as silence
         float *dst = vv + (int64_t)utt * ws_stride + (int64_t)b * ob;
         for (int i = t; i < n_left; i += CT) dst[i] = 0.f;
     }
+    }   // blocks of the run
 }
 
 constexpr size_t FFT_SMEM = sizeof(float2) * SM_POINTS;
@@ -792,7 +850,8 @@ int launch_convolve_finish(AugCtx *ctx, const float *speech, int64_t stride, con
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FFT2_SMEM));
         // every block yields the F2 - (taps - 1) outputs that see no wrap-around, cut to a multiple of 4
         const int ob = (F2 - c.rir_taps + 1) & ~3;
-        dim3 grid2((max_len + ob - 1) / ob, B);
+        const int nblk2 = (max_len + ob - 1) / ob;
+        dim3 grid2((nblk2 + CONV_RUN - 1) / CONV_RUN, B);
         convolve_fused2_kernel<<<grid2, CT, FFT2_SMEM, ctx->stream>>>(
             speech, stride, lengths, bank, bank_len, table, c.max_sources, ctx->hspec, ctx->tw,
             ctx->ys, ctx->vv, ctx->ws_stride, ctx->energy, ctx->status, max_len, ob);

@@ -91,20 +91,25 @@ __device__ __forceinline__ float compress(float e, float floor_v, int mode) {
 // ---------------------------------------------------------------- tile transform
 // Power spectra of `nf` frames starting `hop` apart in `chunk` (shared memory)
 // into ptile[f][k], k <= K/2 (row stride K/2+1).
-template <int K, int E>
-__device__ __forceinline__ void tile_power(const float *chunk, int nf, int win, int hop,
-                                           float2 *fbuf, float *ptile,
-                                           const float2 *__restrict__ tw) {
-    static_assert(K / E == GROUP, "one FFT per 64-thread group");
-    const int tid = threadIdx.x, tg = tid & (GROUP - 1), grp = tid / GROUP;
-    float2 *s = fbuf + grp * padded_points(K);
-    constexpr int NBP = K / 2 + 1;
-    float wv[E];
+// Window values of the E points a thread holds (n = tg + GROUP r), zero beyond the window.
+template <int E>
+__device__ __forceinline__ void window_values(float *wv, int win) {
+    const int tg = threadIdx.x & (GROUP - 1);
 #pragma unroll
     for (int r = 0; r < E; ++r) {
         const int n = tg + GROUP * r;
         wv[r] = n < win ? 0.5f - 0.5f * cospif(2.f * (float)n / (float)win) : 0.f;
     }
+}
+
+template <int K, int E>
+__device__ __forceinline__ void tile_power(const float *chunk, int nf, int win, int hop,
+                                           const float *wv, float2 *fbuf, float *ptile,
+                                           const float2 *__restrict__ tw) {
+    static_assert(K / E == GROUP, "one FFT per 64-thread group");
+    const int tid = threadIdx.x, tg = tid & (GROUP - 1), grp = tid / GROUP;
+    float2 *s = fbuf + grp * padded_points(K);
+    constexpr int NBP = K / 2 + 1;
     const GroupSync gsync{grp + 1, GROUP};
     const int npair = (nf + 1) / 2;
     const int iters = (npair + NGROUP - 1) / NGROUP;
@@ -156,27 +161,33 @@ __device__ __forceinline__ void tile_power(const float *chunk, int nf, int win, 
 #ifndef FEAT_FT_1024
 #define FEAT_FT_1024 16     // frames per CTA tile, 1024-point transform
 #endif
+#ifndef FEAT_TILES
+#define FEAT_TILES 4        // consecutive tiles one CTA works through
+#endif
 template <int K>
 struct Plan;
 template <>
 struct Plan<512> {
-    static constexpr int E = 8, FT = FEAT_FT_512;
+    static constexpr int E = 8, FT = FEAT_FT_512, TILES = FEAT_TILES;
 };
 template <>
 struct Plan<1024> {
-    static constexpr int E = 16, FT = FEAT_FT_1024;
+    static constexpr int E = 16, FT = FEAT_FT_1024, TILES = FEAT_TILES;
 };
 
+#ifndef FEAT_MINB
+#define FEAT_MINB 3           // CTAs per SM the register budget is set for
+#endif
 // MODE 0: wave -> power (global).  MODE 1: y_s + g v -> features.
 template <int K, int MODE>
-__global__ void __launch_bounds__(FEAT_THREADS)
+__global__ void __launch_bounds__(FEAT_THREADS, FEAT_MINB)
 frames_kernel(const float *__restrict__ in_a, const float *__restrict__ in_b, int64_t in_stride,
               const float *__restrict__ gain, const AugUttParams *__restrict__ table,
               const int *__restrict__ lengths, int win, int hop, int M, int T_max,
               const aug::MelBin *__restrict__ melw, const int *__restrict__ melstart,
               const float2 *__restrict__ tw, float floor_v, float pad_v, int comp,
               float *__restrict__ out, int *__restrict__ counts, int n_cap) {
-    constexpr int E = Plan<K>::E, FT = Plan<K>::FT, NBP = K / 2 + 1;
+    constexpr int E = Plan<K>::E, FT = Plan<K>::FT, TILES = Plan<K>::TILES, NBP = K / 2 + 1;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float2 *fbuf = reinterpret_cast<float2 *>(smem_raw);            // [NGROUP][K + K/8]
     float *ptile = reinterpret_cast<float *>(fbuf + NGROUP * padded_points(K));    // [FT][NBP]
@@ -185,76 +196,110 @@ frames_kernel(const float *__restrict__ in_a, const float *__restrict__ in_b, in
     aug::MelBin *mw = reinterpret_cast<aug::MelBin *>(chunk + chunk_cap);   // [NBP]
     int *mst = reinterpret_cast<int *>(mw + NBP + 1);                       // [M+2]
 
-    const int utt = blockIdx.y, t0 = blockIdx.x * FT, tid = threadIdx.x;
+    const int utt = blockIdx.y, tid = threadIdx.x;
+    const int run0 = blockIdx.x * (FT * TILES);    // first frame of this CTA's run of tiles
     const int N = min(max(lengths[utt], 0), n_cap);
     const int T = min(frame_count(N, win, hop), T_max);
     if (blockIdx.x == 0 && tid == 0) counts[utt] = T;
-    const int rows = min(FT, T_max - t0);          // rows of the output this tile owns
+    const int rows = min(FT * TILES, T_max - run0);     // rows of the output this run owns
     if (rows <= 0) return;
-    const int nf = max(0, min(FT, T - t0));        // of which real frames
+    const int nfr = max(0, min(FT * TILES, T - run0));  // of which real frames
     const int out_w = MODE == 0 ? NBP : M;
-    float *orow = out + ((int64_t)utt * T_max + t0) * out_w;
+    float *orun = out + ((int64_t)utt * T_max + run0) * out_w;
     const float fill = MODE == 0 ? 0.f : pad_v;
-    for (int i = nf * out_w + tid; i < rows * out_w; i += FEAT_THREADS) orow[i] = fill;
-    if (nf == 0) return;
+    for (int i = nfr * out_w + tid; i < rows * out_w; i += FEAT_THREADS) orun[i] = fill;
+    if (nfr == 0) return;
 
-    // stage the samples of these frames
-    const int s0 = t0 * hop;
-    const int ns = (nf - 1) * hop + win;
-    const float *pa = in_a + (int64_t)utt * in_stride + s0;
+    const float g = MODE == 1 ? gain[utt] : 0.f;
+    const float *ra = in_a + (int64_t)utt * in_stride;
+    const float *rb = MODE == 1 ? in_b + (int64_t)utt * in_stride : nullptr;
+    const bool vec = (hop & 3) == 0 && (in_stride & 3) == 0;
     if (MODE == 1) {
-        const float g = gain[utt];
-        const float *pb = in_b + (int64_t)utt * in_stride + s0;
-        if ((hop & 3) == 0) {
-            for (int i = tid * 4; i < ns; i += FEAT_THREADS * 4) {
-                // rows are zero- or garbage-padded up to a multiple of 4 floats but always allocated
-                const float4 x = *reinterpret_cast<const float4 *>(pa + i);
-                float4 y = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (g != 0.f) y = *reinterpret_cast<const float4 *>(pb + i);
-                *reinterpret_cast<float4 *>(chunk + i) = make_float4(
-                    fmaf(g, y.x, x.x), fmaf(g, y.y, x.y), fmaf(g, y.z, x.z), fmaf(g, y.w, x.w));
-            }
-        } else {
-            for (int i = tid; i < ns; i += FEAT_THREADS)
-                chunk[i] = g != 0.f ? fmaf(g, pb[i], pa[i]) : pa[i];
-        }
         for (int k = tid; k < NBP; k += FEAT_THREADS) mw[k] = melw[(int64_t)utt * NBP + k];
         for (int m = tid; m < M + 2; m += FEAT_THREADS) mst[m] = melstart[(int64_t)utt * (M + 2) + m];
-    } else {
-        if ((hop & 3) == 0 && (in_stride & 3) == 0) {
-            for (int i = tid * 4; i < ns; i += FEAT_THREADS * 4) {
-                if (s0 + i + 3 < N) {
-                    *reinterpret_cast<float4 *>(chunk + i) = *reinterpret_cast<const float4 *>(pa + i);
-                } else {
-                    for (int j = 0; j < 4; ++j) chunk[i + j] = (s0 + i + j < N) ? pa[i + j] : 0.f;
+    }
+    float wv[E];
+    window_values<E>(wv, win);
+
+    for (int tile = 0; tile < TILES; ++tile) {
+        const int t0 = run0 + tile * FT;
+        const int nf = min(FT, T - t0);                 // frames of this tile
+        if (nf <= 0) break;
+        const int s0 = t0 * hop;
+        const int ns = (nf - 1) * hop + win;            // samples they cover (all below N)
+        const float *pa = ra + s0;
+        const float *pb = MODE == 1 ? rb + s0 : nullptr;
+
+        // Stage the samples of these frames.  All loads of a batch are issued before
+        // the first is used: a tile costs one memory round trip, not one per 1024
+        // samples.  The stretch of the next tile is pulled into L2 meanwhile.
+        if (vec) {
+            constexpr int SB = 6;                       // 128-bit loads per thread, array and batch
+            for (int i0 = tid * 4; i0 < ns; i0 += SB * FEAT_THREADS * 4) {
+                float4 xa[SB], xb[SB];
+#pragma unroll
+                for (int u = 0; u < SB; ++u) {
+                    const int i = i0 + u * FEAT_THREADS * 4;
+                    xa[u] = xb[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    // rows are allocated up to a multiple of 4 floats: whole groups can be read
+                    if (i < ns) {
+                        xa[u] = __ldg(reinterpret_cast<const float4 *>(pa + i));
+                        if (MODE == 1 && g != 0.f) xb[u] = __ldg(reinterpret_cast<const float4 *>(pb + i));
+                    }
+                }
+                if (i0 == tid * 4 && tile + 1 < TILES && t0 + FT < T) {
+                    // next tile: FT hop samples further on, 128 bytes per prefetch
+                    const int nxt = s0 + FT * hop + tid * 32;
+                    if (nxt < N) {
+                        asm volatile("prefetch.global.L2 [%0];" ::"l"(ra + nxt));
+                        if (MODE == 1 && g != 0.f) asm volatile("prefetch.global.L2 [%0];" ::"l"(rb + nxt));
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < SB; ++u) {
+                    const int i = i0 + u * FEAT_THREADS * 4;
+                    if (i < ns) {
+                        float4 x = xa[u];
+                        const float4 y = xb[u];
+                        if (MODE == 0 && s0 + i + 3 >= N) {      // caller's buffer: nothing beyond N is used
+                            if (s0 + i + 1 >= N) x.y = 0.f;
+                            if (s0 + i + 2 >= N) x.z = 0.f;
+                            x.w = 0.f;
+                        }
+                        *reinterpret_cast<float4 *>(chunk + i) = make_float4(
+                            fmaf(g, y.x, x.x), fmaf(g, y.y, x.y), fmaf(g, y.z, x.z), fmaf(g, y.w, x.w));
+                    }
                 }
             }
         } else {
-            for (int i = tid; i < ns; i += FEAT_THREADS) chunk[i] = pa[i];
-        }
-    }
-    __syncthreads();
-
-    tile_power<K, E>(chunk, nf, win, hop, fbuf, ptile, tw);
-
-    if (MODE == 0) {
-        for (int i = tid; i < nf * NBP; i += FEAT_THREADS) orow[i] = ptile[i];
-    } else {
-        // Filterbank with the lanes of a warp over the frames of the tile: all lanes
-        // of a band walk the same bins (weights are broadcasts, the odd row stride
-        // of ptile keeps the power reads conflict-free, no lane waits for a wider
-        // band).  Results go through shared memory so the global store is contiguous.
-        float *etile = reinterpret_cast<float *>(fbuf);           // [FT][M], transforms are done
-        constexpr int BPW = 32 / FT;                              // bands per warp step
-        const int lane = tid & 31, warp = tid >> 5;
-        const int f = lane % FT, sub = lane / FT;
-        for (int m0 = warp * BPW; m0 < M; m0 += (FEAT_THREADS / 32) * BPW) {
-            const int m = m0 + sub;
-            if (m < M && f < nf)
-                etile[f * M + m] = compress(band_energy(ptile + f * NBP, mw, mst, m), floor_v, comp);
+            for (int i = tid; i < ns; i += FEAT_THREADS)
+                chunk[i] = (MODE == 1 && g != 0.f) ? fmaf(g, pb[i], pa[i]) : pa[i];
         }
         __syncthreads();
-        for (int i = tid; i < nf * M; i += FEAT_THREADS) orow[i] = etile[i];
+
+        tile_power<K, E>(chunk, nf, win, hop, wv, fbuf, ptile, tw);
+
+        float *orow = orun + (int64_t)tile * FT * out_w;
+        if (MODE == 0) {
+            for (int i = tid; i < nf * NBP; i += FEAT_THREADS) orow[i] = ptile[i];
+        } else {
+            // Filterbank with the lanes of a warp over the frames of the tile: all lanes
+            // of a band walk the same bins (weights are broadcasts, the odd row stride
+            // of ptile keeps the power reads conflict-free, no lane waits for a wider
+            // band).  Results go through shared memory so the global store is contiguous.
+            float *etile = reinterpret_cast<float *>(fbuf);           // [FT][M], transforms are done
+            constexpr int BPW = 32 / FT;                              // bands per warp step
+            const int lane = tid & 31, warp = tid >> 5;
+            const int f = lane % FT, sub = lane / FT;
+            for (int m0 = warp * BPW; m0 < M; m0 += (FEAT_THREADS / 32) * BPW) {
+                const int m = m0 + sub;
+                if (m < M && f < nf)
+                    etile[f * M + m] = compress(band_energy(ptile + f * NBP, mw, mst, m), floor_v, comp);
+            }
+            __syncthreads();
+            for (int i = tid; i < nf * M; i += FEAT_THREADS) orow[i] = etile[i];
+        }
+        __syncthreads();   // ptile, etile (= the transform buffers) and chunk are reused by the next tile
     }
 }
 
@@ -297,7 +342,8 @@ int launch_frames(AugCtx *ctx, const float *a, const float *b, int64_t stride, c
     if (smem > 227 * 1024) return AUG_ECAP;
     AUG_CUDA_OK(cudaFuncSetAttribute(frames_kernel<K, MODE>,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    dim3 grid((T_max + FT - 1) / FT, B);
+    constexpr int RUN = FT * Plan<K>::TILES;
+    dim3 grid((T_max + RUN - 1) / RUN, B);
     frames_kernel<K, MODE><<<grid, FEAT_THREADS, smem, ctx->stream>>>(
         a, b, stride, ctx->gain, table, lengths, c.win, c.hop, c.n_mel, T_max, ctx->melw,
         ctx->melstart, ctx->tw, c.log_floor, c.pad_value, c.compression, out, counts,

@@ -198,12 +198,14 @@ __device__ __forceinline__ void pass_pair(float2 *a, float2 *b, int t, const flo
                                           Sync sync) {
     constexpr int NB = E / R;
     float2 v[NB][R];
-    gather<N, E, R, NS_PREV>(v, a, t);
-    sync();
-    pass_from_regs<N, E, R, NS>(v, a, t, tw);
-    gather<N, E, R, NS_PREV>(v, b, t);
-    sync();
-    pass_from_regs<N, E, R, NS>(v, b, t, tw);
+    // not unrolled: the second transform reuses the first one's instructions
+#pragma unroll 1
+    for (int h = 0; h < 2; ++h) {
+        float2 *s = h ? b : a;
+        gather<N, E, R, NS_PREV>(v, s, t);
+        sync();
+        pass_from_regs<N, E, R, NS>(v, s, t, tw);
+    }
 }
 
 struct CtaSync {

@@ -103,9 +103,14 @@ extern "C" int aug_sample_params(uint64_t seed, const AugDist *dist, int B, cons
             if (hi > dist->bank_len) hi = dist->bank_len;
             int64_t lo = hi / 2 > dist->min_noise_len ? hi / 2 : dist->min_noise_len;
             if (lo > hi) lo = hi;
-            const int64_t len = rng.integer(lo, hi);
+            int64_t len = rng.integer(lo, hi);
+            int64_t off = rng.integer(0, dist->bank_len - len);
+            if (len >= 4) {   // whole groups of four samples from a 16-byte boundary: 128-bit loads
+                len &= ~(int64_t)3;
+                off &= ~(int64_t)3;
+            }
             r.noise_len[j] = (int32_t)len;
-            r.noise_offset[j] = rng.integer(0, dist->bank_len - len);
+            r.noise_offset[j] = off;
             r.noise_weight[j] = 1.f;
         }
         table_host[b] = r;

@@ -154,9 +154,11 @@ def _place(rng, room, others, margin=0.3, min_dist=0.5):
 
 
 def sample_table(rng, lengths, bank_len, *, room_lo, room_hi, t60, order,
-                 n_noise, snr, alpha, min_noise_len=4000) -> np.ndarray:
+                 n_noise, snr, alpha, min_noise_len=4000, noise_align=4) -> np.ndarray:
     """Draw one table row per utterance.  Ranges are (lo, hi) pairs; a pair with
-    lo == hi gives a constant."""
+    lo == hi gives a constant.  Noise stretches start and end on multiples of
+    `noise_align` samples (4 = 16 bytes, what a sampler that cares about load width
+    hands out; 1 = anywhere)."""
     B = len(lengths)
     tab = np.zeros(B, dtype=UTT_DTYPE)
     for b in range(B):
@@ -182,8 +184,12 @@ def sample_table(rng, lengths, bank_len, *, room_lo, room_hi, t60, order,
             lo = max(min_noise_len, hi // 2)
             ln = int(rng.integers(lo, hi + 1))
             ln = min(ln, bank_len)
+            off = int(rng.integers(0, bank_len - ln + 1))
+            if noise_align > 1:
+                ln = max(noise_align, ln // noise_align * noise_align)
+                off = off // noise_align * noise_align
             row["noise_len"][j] = ln
-            row["noise_offset"][j] = int(rng.integers(0, bank_len - ln + 1))
+            row["noise_offset"][j] = off
             row["noise_weight"][j] = 1.0
     return tab
 
@@ -219,7 +225,8 @@ _RECIPES = {
 
 def make_workload(index: int, seed: int = 0, *, batch: Optional[int] = None,
                   dur_scale: float = 1.0, bank_seconds: Optional[float] = None,
-                  taps: Optional[int] = None, order: Optional[int] = None) -> Workload:
+                  taps: Optional[int] = None, order: Optional[int] = None,
+                  noise_align: int = 4) -> Workload:
     """Workload `index` (1..5).  `batch`, `dur_scale`, `taps`, `order` shrink a
     workload for checks the slow CPU implementation must finish; the defaults
     are the full sizes."""
@@ -249,7 +256,7 @@ def make_workload(index: int, seed: int = 0, *, batch: Optional[int] = None,
     ordr = r["order"] if order is None else int(order)
     table = sample_table(rng, lengths, bank.shape[0], room_lo=r["room_lo"], room_hi=r["room_hi"],
                          t60=r["t60"], order=ordr, n_noise=r["n_noise"], snr=r["snr"],
-                         alpha=r["alpha"])
+                         alpha=r["alpha"], noise_align=noise_align)
     cfg = dict(_COMMON)
     cfg.update(n_mel=r["n_mel"], n_fft=r["n_fft"], max_order=ordr,
                rir_taps=r["taps"] if taps is None else int(taps))

@@ -136,6 +136,22 @@ def test_pipeline_matches_oracle(index):
     print(f"config{index} reduced: worst log-mel err {worst_f:.2e}, worst wave err/rms {worst_w:.2e}")
 
 
+@pytest.mark.parametrize("index", [2, 4, 3])
+def test_pipeline_with_unaligned_and_very_short_noise_stretches(index):
+    """Noise stretches that start anywhere and have any length (the 128-bit load path
+    needs multiples of four samples), down to loops of a few samples."""
+    w = small(index, **dict(REDUCED[index], batch=4), noise_align=1)
+    tab = w.table
+    assert any(int(o) % 4 for o in tab["noise_offset"][:, 0]) or any(int(n) % 4 for n in tab["noise_len"][:, 0])
+    tab["noise_offset"][0, 0], tab["noise_len"][0, 0] = 1001, 3        # shorter than one load
+    tab["noise_offset"][1, 0], tab["noise_len"][1, 0] = 2002, 1031     # wraps many times per block
+    tab["noise_offset"][2, 0], tab["noise_len"][2, 0] = 4000, 4100     # aligned start, unaligned length
+    dev = Device(w)
+    F, counts, wave = dev.pipeline(want_wave=True)
+    assert dev.ctx.aug_last_status() == (-1, 0)
+    check_pipeline_against_oracle(dev, F, counts, wave, oracle_batch(w))
+
+
 def test_pipeline_edge_lengths_and_no_noise():
     w = small(2, batch=8, dur_scale=0.12)
     w.lengths[:6] = [0, 1, 399, 400, 559, 560]
