@@ -10,7 +10,7 @@
 // The filterbank is applied as a gather: band m sums the bins of edge interval m
 // with their rising weights and those of interval m+1 with their falling
 // weights; the intervals are contiguous bin ranges because the warp of Eq. 1 is
-// monotone.
+// monotone.  The fused kernel walks every interval once and keeps both sums.
 #include "common.cuh"
 #include "fft.cuh"
 
@@ -175,6 +175,14 @@ struct Plan<1024> {
     static constexpr int E = 16, FT = FEAT_FT_1024, TILES = FEAT_TILES;
 };
 
+// Floats of the region that first holds the transform buffers of the four groups and
+// then, once a tile's transforms are done, the two interval sums [FT][M+1] of the filterbank.
+template <int K>
+__host__ __device__ constexpr int fbuf_floats(int FT, int M) {
+    const int a = 2 * NGROUP * padded_points(K), b = 2 * FT * (M + 1);
+    return ((a > b ? a : b) + 3) & ~3;
+}
+
 #ifndef FEAT_MINB
 #define FEAT_MINB 3           // CTAs per SM the register budget is set for
 #endif
@@ -189,8 +197,8 @@ frames_kernel(const float *__restrict__ in_a, const float *__restrict__ in_b, in
               float *__restrict__ out, int *__restrict__ counts, int n_cap) {
     constexpr int E = Plan<K>::E, FT = Plan<K>::FT, TILES = Plan<K>::TILES, NBP = K / 2 + 1;
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    float2 *fbuf = reinterpret_cast<float2 *>(smem_raw);            // [NGROUP][K + K/8]
-    float *ptile = reinterpret_cast<float *>(fbuf + NGROUP * padded_points(K));    // [FT][NBP]
+    float2 *fbuf = reinterpret_cast<float2 *>(smem_raw);            // [NGROUP][K + K/8]; later the interval sums
+    float *ptile = reinterpret_cast<float *>(smem_raw) + fbuf_floats<K>(FT, M);    // [FT][NBP]
     float *chunk = ptile + FT * NBP;                                // [(FT-1) hop + win] (+pad)
     const int chunk_cap = ((FT - 1) * hop + win + 3) & ~3;
     aug::MelBin *mw = reinterpret_cast<aug::MelBin *>(chunk + chunk_cap);   // [NBP]
@@ -283,23 +291,42 @@ frames_kernel(const float *__restrict__ in_a, const float *__restrict__ in_b, in
         if (MODE == 0) {
             for (int i = tid; i < nf * NBP; i += FEAT_THREADS) orow[i] = ptile[i];
         } else {
-            // Filterbank with the lanes of a warp over the frames of the tile: all lanes
-            // of a band walk the same bins (weights are broadcasts, the odd row stride
-            // of ptile keeps the power reads conflict-free, no lane waits for a wider
-            // band).  Results go through shared memory so the global store is contiguous.
-            float *etile = reinterpret_cast<float *>(fbuf);           // [FT][M], transforms are done
-            constexpr int BPW = 32 / FT;                              // bands per warp step
+            // Filterbank with the lanes of a warp over the frames of the tile and one edge
+            // interval per lane group: the bins of interval j are walked once, giving
+            // both their rising sum (band j) and their falling sum (band j-1); all lanes
+            // of an interval walk the same bins (weights are broadcasts, the odd row
+            // strides keep the other accesses conflict-free, no lane waits for a wider
+            // band).  Band m = rising sum of interval m + falling sum of interval m+1,
+            // added while the results are written out contiguously.
+            float *up_s = reinterpret_cast<float *>(fbuf);            // [FT][M+1], transforms are done
+            float *dn_s = up_s + FT * (M + 1);                        // [FT][M+1]
+            const float2 *mw2 = reinterpret_cast<const float2 *>(mw);
+            constexpr int BPW = 32 / FT;                              // intervals per warp step
             const int lane = tid & 31, warp = tid >> 5;
             const int f = lane % FT, sub = lane / FT;
-            for (int m0 = warp * BPW; m0 < M; m0 += (FEAT_THREADS / 32) * BPW) {
-                const int m = m0 + sub;
-                if (m < M && f < nf)
-                    etile[f * M + m] = compress(band_energy(ptile + f * NBP, mw, mst, m), floor_v, comp);
+            for (int j0 = warp * BPW; j0 <= M; j0 += (FEAT_THREADS / 32) * BPW) {
+                const int j = j0 + sub;
+                if (j <= M && f < nf) {
+                    const float *p = ptile + f * NBP;
+                    float u = 0.f, d = 0.f;
+                    const int k1 = mst[j + 1];
+                    for (int k = mst[j]; k < k1; ++k) {
+                        const float2 w = mw2[k];
+                        const float pk = p[k];
+                        u = fmaf(w.x, pk, u);
+                        d = fmaf(w.y, pk, d);
+                    }
+                    up_s[f * (M + 1) + j] = u;
+                    dn_s[f * (M + 1) + j] = d;
+                }
             }
             __syncthreads();
-            for (int i = tid; i < nf * M; i += FEAT_THREADS) orow[i] = etile[i];
+            for (int i = tid; i < nf * M; i += FEAT_THREADS) {
+                const int ff = i / M, m = i - ff * M;
+                orow[i] = compress(up_s[ff * (M + 1) + m] + dn_s[ff * (M + 1) + m + 1], floor_v, comp);
+            }
         }
-        __syncthreads();   // ptile, etile (= the transform buffers) and chunk are reused by the next tile
+        __syncthreads();   // ptile, the interval sums (= the transform buffers) and chunk are reused by the next tile
     }
 }
 
@@ -336,7 +363,7 @@ int launch_frames(AugCtx *ctx, const float *a, const float *b, int64_t stride, c
     const AugConfig &c = ctx->cfg;
     constexpr int FT = Plan<K>::FT, NBP = K / 2 + 1;
     const int chunk_cap = ((FT - 1) * c.hop + c.win + 3) & ~3;
-    const size_t smem = sizeof(float2) * NGROUP * padded_points(K) + sizeof(float) * FT * NBP +
+    const size_t smem = sizeof(float) * fbuf_floats<K>(FT, c.n_mel) + sizeof(float) * FT * NBP +
                         sizeof(float) * chunk_cap + sizeof(aug::MelBin) * (NBP + 1) +
                         sizeof(int) * (c.n_mel + 2);
     if (smem > 227 * 1024) return AUG_ECAP;
