@@ -64,16 +64,20 @@ def conv_work(w):
     """Nominal flops and compulsory bytes of the convolution step for one batch, per kernel.
     Per source one forward real FFT per block (2.5 F log2 F), 8 flops per bin and
     partition for the spectral multiply, two inverse FFTs per block (one without
-    noise).  Responses of up to 4096 / 8192 taps take one partition of an 8192- /
-    16384-point transform and a single fused kernel does all of it (bytes: inputs
-    read once, y_s and v written once, response spectra read once); longer ones are
-    cut into 4096-tap partitions: block_spectra_kernel does the forward FFTs (inputs
-    in, block spectra out) and spectral_convolve_kernel the rest (block and partition
-    spectra in, y_s and v out)."""
+    noise).  Responses of up to 8192 taps take one partition of a 16384-point
+    transform and a block yields 16384 - taps + 1 outputs (cut to a multiple of 4): a
+    single fused kernel does all of it (bytes: inputs read once, y_s and v written
+    once, response spectra read once).  Longer ones are cut into 4096-tap partitions
+    of an 8192-point transform with 4096 outputs per block: block_spectra_kernel does
+    the forward FFTs (inputs in, block spectra out) and spectral_convolve_kernel the
+    rest (block and partition spectra in, y_s and v out)."""
     taps = int(w.cfg["rir_taps"])
-    blk = 8192 if 4096 < taps <= 8192 else 4096
-    F = 2 * blk
-    P = -(-taps // blk)
+    if taps <= 8192:
+        F, P = 16384, 1
+        blk = (F - taps + 1) & ~3
+    else:
+        F, blk = 8192, 4096
+        P = -(-taps // blk)
     fft = 2.5 * F * np.log2(F)
     spec = (F // 2) * 8.0
     fwd_f = fwd_b = fin_f = fin_b = 0.0
