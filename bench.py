@@ -431,6 +431,29 @@ def run_ours(args):
     barrier()
     h2d, d2h = ctx.aug_last_host_bytes()     # what the library really copied (ragged rows)
 
+    # ---- the same with the noise bank uploaded once (a noise database does not change
+    # from batch to batch): only speech, lengths and the table cross the bus every step
+    dt_res, h2d_res = 0.0, 0
+    if not args.skip_e2e:
+        ctx.aug_upload_noise_bank(bk_h, w.bank.size)
+
+        def step_res():
+            ctx.aug_pipeline_host(sp_h, w.stride, ln_h, None, w.bank.size, tb_h, w.B, f_h, T_max, c_h)
+
+        step_res()
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            step_res()
+        torch.cuda.synchronize()
+        dt_res = time.perf_counter() - t0
+        barrier()
+        h2d_res, _ = ctx.aug_last_host_bytes()
+
+    if world > 1:
+        t_res = torch.tensor([dt_res], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t_res, op=dist.ReduceOp.MAX)
+        dt_res = float(t_res.cpu()[0])
     audio_total, ms_total, dt_e2e = combine_ranks(w.audio_seconds, ms_total, dt_e2e, world, "cuda")
     value = audio_total * args.steps / (ms_total * 1e-3)
     e2e_value = audio_total * e2e_steps / dt_e2e
@@ -504,6 +527,12 @@ def run_ours(args):
             "roofline": roofline,
             "cpu_baseline": {"value": cpu_val, "unit": UNIT, "cores": cores, "kind": "oracle",
                              "sample": cpu_sample}}
+    if dt_res > 0:
+        line["e2e_resident_bank"] = {"value": audio_total * e2e_steps / dt_res, "unit": UNIT,
+                                     "h2d_bytes_per_step": h2d_res, "d2h_bytes_per_step": d2h,
+                                     "steps": e2e_steps,
+                                     "note": "noise bank uploaded once with aug_upload_noise_bank; "
+                                             "e2e above sends it with every step"}
     if args.cpu_fast_utts > 0:
         fv, fs_, fw = time_fast_cpu(w, args.cpu_fast_utts)
         line["cpu_fast"] = {"value": fv, "unit": UNIT, "cores": fw, "kind": "numpy/scipy FFT pipeline",

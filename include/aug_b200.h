@@ -292,11 +292,26 @@ int aug_pipeline(AugCtx *ctx, const float *speech_dev, int64_t speech_stride,
  * again.  Internally the batch is cut into up to 8 chunks of utterances that are
  * copied in, computed and copied out concurrently on three streams; speech rows
  * are copied only up to their length when that saves more than the extra copy
- * calls cost.  Host buffers should be pinned for full copy bandwidth. */
+ * calls cost.  Host buffers should be pinned: copies then run asynchronously, and
+ * the ragged rows of a pinned (mapped) speech buffer are fetched by one small kernel
+ * per chunk that reads host memory directly instead of one copy per row.
+ * noise_bank_host may be NULL with bank_len > 0
+ * when a bank of exactly bank_len samples was uploaded with aug_upload_noise_bank:
+ * that copy is then used and nothing of the bank crosses the bus (AUG_EINVAL if
+ * there is none or its length differs). */
 int aug_pipeline_host(AugCtx *ctx, const float *speech_host, int64_t speech_stride,
                       const int *lengths_host, const float *noise_bank_host, int64_t bank_len,
                       const AugUttParams *table_host, int B, float *feats_host, int T_max,
                       int *frame_counts_host);
+
+/* A noise database that stays the same from batch to batch need not be sent with
+ * every aug_pipeline_host call: copy bank_len samples into the context's device
+ * staging once (host_staging contexts only, bank_len <= max_bank_samples; the call
+ * synchronises, so the host buffer is free on return).  The copy stays valid until
+ * the next aug_upload_noise_bank or the next aug_pipeline_host call that passes a
+ * bank pointer of its own.  (Interface of this library; the paper's example servers
+ * keep their noise database in host memory.) */
+int aug_upload_noise_bank(AugCtx *ctx, const float *noise_bank_host, int64_t bank_len);
 
 /* -------------------------------------------------------------- measurement utilities
  * (instrumentation of this library; the paper has no counterpart) */

@@ -83,6 +83,7 @@ struct AugCtx {
     int64_t last_h2d, last_d2h;                // bytes the last aug_pipeline_host call copied
     cudaStream_t s_h2d, s_d2h;                 // copy streams of the host-buffer entry point
     cudaEvent_t ev_in[aug::HOST_CHUNKS], ev_out[aug::HOST_CHUNKS], ev_start;
+    int64_t bank_resident;                     // samples of st_bank filled by aug_upload_noise_bank (0 = none)
 };
 
 #define AUG_CUDA_OK(expr)                         \

@@ -192,6 +192,59 @@ def test_host_buffer_entry_point_matches_device_one():
     assert np.max(np.abs(Fh - F.cpu().numpy())) < 1e-3
 
 
+def test_host_entry_point_from_pinned_memory_matches_pageable():
+    """Ragged rows of a pinned batch are fetched by a kernel that reads host memory
+    directly; pageable memory goes through one copy per row.  Same features either way."""
+    import torch
+    w = small(2, batch=12, dur_scale=0.5)
+    w.lengths[3] = 0
+    w.lengths[4] = 1
+    dev = Device(w, host_staging=True)
+    tab = np.ascontiguousarray(w.table)
+    Fp = np.full((w.B, dev.T_max, dev.M), np.nan, dtype=np.float32)
+    cp = np.full(w.B, -1, dtype=np.int32)
+    dev.ctx.aug_pipeline_host(w.speech, w.stride, w.lengths, w.bank, w.bank.size, tab, w.B, Fp, dev.T_max, cp)
+    pin = lambda a: torch.from_numpy(a).pin_memory()
+    Fh, ch = torch.full((w.B, dev.T_max, dev.M), float("nan")).pin_memory(), torch.full((w.B,), -1, dtype=torch.int32).pin_memory()
+    dev.ctx.aug_pipeline_host(pin(w.speech), w.stride, pin(w.lengths), pin(w.bank), w.bank.size,
+                              pin(tab.view(np.uint8).reshape(-1).copy()), w.B, Fh, dev.T_max, ch)
+    assert np.array_equal(ch.numpy(), cp)
+    assert list(cp[3:5]) == [0, 0]
+    assert np.max(np.abs(Fh.numpy() - Fp)) < 1e-3
+    F, counts, _ = dev.pipeline(want_wave=False)
+    assert np.array_equal(counts.cpu().numpy(), cp) and np.max(np.abs(F.cpu().numpy() - Fp)) < 1e-3
+
+
+def test_host_entry_point_with_an_uploaded_noise_bank():
+    """A bank uploaded once serves later calls that pass no bank pointer; results and the
+    bytes copied say so; a call with a bank of its own replaces the uploaded one."""
+    w = small(2, batch=20, dur_scale=0.1)
+    dev = Device(w, host_staging=True)
+    args = (w.speech, w.stride, w.lengths)
+    tab = np.ascontiguousarray(w.table)
+    outs = []
+    for use_resident in (False, True, True):
+        Fh = np.full((w.B, dev.T_max, dev.M), np.nan, dtype=np.float32)
+        ch = np.full(w.B, -1, dtype=np.int32)
+        if use_resident and not outs[1:]:
+            dev.ctx.aug_upload_noise_bank(w.bank, w.bank.size)
+        dev.ctx.aug_pipeline_host(*args, None if use_resident else w.bank, w.bank.size, tab, w.B, Fh,
+                                  dev.T_max, ch)
+        outs.append((Fh, ch, dev.ctx.aug_last_host_bytes()[0]))
+    assert np.array_equal(outs[0][1], outs[1][1]) and np.array_equal(outs[0][1], outs[2][1])
+    # (the impulse responses are summed with atomics: runs differ in the last bits)
+    assert np.max(np.abs(outs[0][0] - outs[1][0])) < 1e-3 and np.max(np.abs(outs[0][0] - outs[2][0])) < 1e-3
+    assert outs[0][2] - outs[1][2] == 4 * w.bank.size
+    # without an upload of that length there is nothing to use
+    assert dev.ctx.aug_pipeline_host(*args, None, w.bank.size - 4, tab, w.B, outs[0][0].copy(), dev.T_max,
+                                     outs[0][1].copy(), check=False) == binding.AUG_EINVAL
+    dev.ctx.aug_pipeline_host(*args, w.bank, w.bank.size, tab, w.B, outs[0][0].copy(), dev.T_max,
+                              outs[0][1].copy())
+    assert dev.ctx.aug_pipeline_host(*args, None, w.bank.size, tab, w.B, outs[0][0].copy(), dev.T_max,
+                                     outs[0][1].copy(), check=False) == binding.AUG_EINVAL
+    assert dev.ctx.aug_upload_noise_bank(w.bank, w.bank.size + 1, check=False) == binding.AUG_ECAP
+
+
 def test_errors_and_status_word():
     w = small(1, batch=2, dur_scale=0.1)
     dev = Device(w)
