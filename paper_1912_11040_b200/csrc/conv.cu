@@ -1,24 +1,32 @@
-// Step 2: reverberation by partitioned FFT overlap convolution, noise mixing.
+// Step 2: reverberation by FFT overlap convolution, noise mixing.
 //
-// The impulse response is cut into partitions of CONV_BLK taps whose spectra are
-// computed once per batch (rir_spectra_kernel).  One CTA then produces one block
-// of CONV_BLK output samples: Y_b = sum_p X_{b-p} H_p, where X_j is the spectrum of
-// the 2*CONV_BLK input samples that end with block j.  Taking each input block
-// together with its predecessor is the overlap-add tail sum moved to the input
-// side, so output blocks never exchange data.  All noise sources are summed in
-// the frequency domain: two inverse transforms per block whatever their number.
+// Every route is overlap-save in form: an output block is computed from the input
+// segment that ends with it (the block plus the samples before it that the response
+// reaches back to), which is the overlap-add tail sum moved to the input side, so
+// output blocks never exchange data.  The route is fixed by the response length:
 //
-// Two routes, same arithmetic:
-//   one partition   convolve_fused_kernel: transform the input segment, multiply,
-//                   inverse-transform, all in one CTA; nothing but y_s and v is stored.
-//   more partitions block_spectra_kernel stores every X_j once; spectral_convolve_kernel
-//                   reads the P spectra a block needs (mostly from L2), multiply-
-//                   accumulates in registers and inverse-transforms.
+//   up to 8192 taps   convolve_fused2_kernel: ONE partition of a 16384-point real
+//                     transform, 16384 - taps + 1 outputs per block.  A CTA does the
+//                     whole block per source -- forward, multiply, inverse -- and
+//                     nothing but y_s and v is stored.  The 8192-point complex
+//                     transform of the (even, odd) sample pairs runs as two
+//                     4096-point transforms joined by a radix-2 step (second half
+//                     of this file).  Noise sources are summed in the time domain.
+//   longer            partitions of CONV_BLK = 4096 taps of an 8192-point transform,
+//                     Y_b = sum_p X_{b-p} H_p with X_j the spectrum of the 8192
+//                     samples that end with block j: block_spectra_kernel stores
+//                     every X_j once; spectral_convolve_kernel reads the P spectra a
+//                     block needs (mostly from L2), multiply-accumulates in registers
+//                     and inverse-transforms.  Noise sources are summed in the
+//                     frequency domain: two inverse transforms per block.
+//   (convolve_fused_kernel, one partition of the 8192-point transform, is kept
+//   behind the compile-time knob AUG_FUSED16K_MIN_TAPS.)
 //
 // A real transform of F points is a complex transform of F/2 points on (even, odd)
-// sample pairs followed by the usual split; thread t owns the bin pairs
-// (k, F/2-k), k = t + 256 q.  Spectra are stored as F/2 complex numbers with the two
-// real bins (0 and F/2) packed into slot 0.
+// sample pairs followed by the usual split; in the 8192-point routes thread t owns
+// the bin pairs (k, F/2-k), k = t + 256 q.  Spectra are stored as F/2 complex numbers
+// with the two real bins (0 and F/2) packed into slot 0; the partition spectra of
+// the responses carry the noise weight and the 1/F of the inverse.
 #include "common.cuh"
 #include "fft.cuh"
 

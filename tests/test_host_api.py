@@ -164,3 +164,21 @@ def test_compute_calls_refuse_without_a_gpu():
     w = synth.make_workload(1, batch=1, dur_scale=0.1)
     with pytest.raises(RuntimeError):
         binding.AugContext(binding.make_config(w.cfg, 1, w.stride))
+
+
+def test_workspace_follows_the_convolution_route():
+    """Responses of up to 8192 taps are convolved without stored block spectra, longer
+    ones with them: the workspace a context asks for shows which route it will take."""
+    w = synth.make_workload(2, batch=2, dur_scale=0.1)
+    sizes = {}
+    for taps in (1, 4096, 4097, 8192, 8193, 24576):
+        cfg = binding.make_config(dict(w.cfg, rir_taps=taps), 64, 160000)
+        sizes[taps] = binding.aug_workspace_bytes(cfg)
+        assert sizes[taps] > 0
+    spectrum = 64 * cfg.max_sources * 8192 * 8              # one 16384-point spectrum per source
+    assert sizes[1] - 64 * cfg.max_sources * 4 * 1 == sizes[8192] - 64 * cfg.max_sources * 4 * 8192
+    blocks = -(-160000 // 4096)
+    extra = sizes[8193] - sizes[8192]
+    assert extra >= 64 * cfg.max_sources * blocks * 4096 * 8   # block spectra of every source
+    assert extra >= spectrum // 2                              # and a third partition
+    assert sizes[24576] > sizes[8193]
