@@ -103,8 +103,7 @@ struct Dft<16> {
 // Powers are built by squaring (w^2, w^4, w^8) and one more product each, so no
 // power is more than three roundings away from the table value.
 template <int R>
-__device__ __forceinline__ void twiddle(float2 *v, float2 w1) {
-    float2 w[R];
+__device__ __forceinline__ void twiddle_powers(float2 *w, float2 w1) {
     w[0] = make_float2(1.f, 0.f);
     w[1] = w1;
 #pragma unroll
@@ -112,6 +111,11 @@ __device__ __forceinline__ void twiddle(float2 *v, float2 w1) {
         const int hi = (r & (r - 1)) ? (r & -r) : r / 2;   // split r = hi + lo with hi a power of two
         w[r] = cmul(w[hi], w[r - hi]);
     }
+}
+template <int R>
+__device__ __forceinline__ void twiddle(float2 *v, float2 w1) {
+    float2 w[R];
+    twiddle_powers<R>(w, w1);
 #pragma unroll
     for (int r = 1; r < R; ++r) v[r] = cmul(v[r], w[r]);
 }
@@ -137,6 +141,23 @@ __device__ __forceinline__ int pad0(int i) { return i; }
 //   v[b][r] = data[(t + b T) + r N/R],  T = N/E threads, b < E/R.
 // Applies the pass twiddles (NS = product of earlier radices), the radix-R DFTs,
 // and scatters the results to `s` in Stockham order.  The caller synchronises.
+// The same pass with the twiddle powers w[r] = w1^r of this thread's (single)
+// butterfly already computed: two transforms that run the same pass side by side
+// share them.
+template <int N, int E, int R, int NS>
+__device__ __forceinline__ void pass_from_regs_tw(float2 (*v)[R], float2 *s, int t, const float2 *w) {
+    static_assert(E == R && NS > 1, "one butterfly per thread, a pass with twiddles");
+    constexpr int PS = out_shift(NS);
+    static_assert(PS >= 0 || NS * R == N, "only the last pass may write the unpadded layout");
+    const int k = t & (NS - 1);
+#pragma unroll
+    for (int r = 1; r < R; ++r) v[0][r] = cmul(v[0][r], w[r]);
+    Dft<R>::run(v[0]);
+    const int base = padi<PS>((t - k) * R + k);
+#pragma unroll
+    for (int r = 0; r < R; ++r) s[base + padi<PS>(r * NS)] = v[0][r];
+}
+
 template <int N, int E, int R, int NS>
 __device__ __forceinline__ void pass_from_regs(float2 (*v)[R], float2 *s, int t,
                                                const float2 *__restrict__ tw) {
@@ -198,6 +219,19 @@ __device__ __forceinline__ void pass_pair(float2 *a, float2 *b, int t, const flo
                                           Sync sync) {
     constexpr int NB = E / R;
     float2 v[NB][R];
+    // one butterfly per thread: both transforms use the same twiddle powers, built once
+    if constexpr (NS > 1 && E == R) {
+        float2 w[R];
+        twiddle_powers<R>(w, __ldg(&tw[tw_index(NS * R, t & (NS - 1))]));
+#pragma unroll 1
+        for (int h = 0; h < 2; ++h) {
+            float2 *s = h ? b : a;
+            gather<N, E, R, NS_PREV>(v, s, t);
+            sync();
+            pass_from_regs_tw<N, E, R, NS>(v, s, t, w);
+        }
+        return;
+    }
     // not unrolled: the second transform reuses the first one's instructions
 #pragma unroll 1
     for (int h = 0; h < 2; ++h) {
