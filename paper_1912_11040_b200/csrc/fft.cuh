@@ -219,10 +219,11 @@ __device__ __forceinline__ void pass_pair(float2 *a, float2 *b, int t, const flo
                                           Sync sync) {
     constexpr int NB = E / R;
     float2 v[NB][R];
-    // one butterfly per thread: both transforms use the same twiddle powers, built once
     if constexpr (NS > 1 && E == R) {
+        // one butterfly per thread: both transforms use the same twiddle powers, built once
         float2 w[R];
         twiddle_powers<R>(w, __ldg(&tw[tw_index(NS * R, t & (NS - 1))]));
+        // not unrolled: the second transform reuses the first one's instructions
 #pragma unroll 1
         for (int h = 0; h < 2; ++h) {
             float2 *s = h ? b : a;
@@ -230,15 +231,14 @@ __device__ __forceinline__ void pass_pair(float2 *a, float2 *b, int t, const flo
             sync();
             pass_from_regs_tw<N, E, R, NS>(v, s, t, w);
         }
-        return;
-    }
-    // not unrolled: the second transform reuses the first one's instructions
+    } else {
 #pragma unroll 1
-    for (int h = 0; h < 2; ++h) {
-        float2 *s = h ? b : a;
-        gather<N, E, R, NS_PREV>(v, s, t);
-        sync();
-        pass_from_regs<N, E, R, NS>(v, s, t, tw);
+        for (int h = 0; h < 2; ++h) {
+            float2 *s = h ? b : a;
+            gather<N, E, R, NS_PREV>(v, s, t);
+            sync();
+            pass_from_regs<N, E, R, NS>(v, s, t, tw);
+        }
     }
 }
 
