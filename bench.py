@@ -124,7 +124,7 @@ def feat_work(w):
 
 # ------------------------------------------------------------------ clocks
 class ClockSampler:
-    def __init__(self, index=0, period=0.02):
+    def __init__(self, index=0, period=0.002):
         self.samples, self.reasons, self.max_mhz = [], set(), None
         self._stop = threading.Event()
         self._thr = None
@@ -546,7 +546,7 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=2, choices=[1, 2, 3, 4, 5])
