@@ -320,6 +320,14 @@ int aug_upload_noise_bank(AugCtx *ctx, const float *noise_bank_host, int64_t ban
                           3 block spectra of the audio (multi-partition responses only),
                           4 convolution, 5 waveform mix (only when requested), 6 features */
 
+/* The fused convolution (responses of up to 8192 taps) sums several noise sources of an
+ * utterance in the frequency domain through parking slots in the workspace, three per
+ * multiprocessor; a CTA that finds none free sums in the time domain instead.
+ * hold != 0 marks every slot taken, so that this second way can be exercised and
+ * timed; hold == 0 frees them.  Synchronises the stream; call it only between
+ * pipeline calls. */
+int aug_hold_parking_slots(AugCtx *ctx, int hold);
+
 /* on != 0: aug_pipeline records CUDA events between its kernels (up to 256 calls
  * are kept); on == 0: stop.  Either way the record is cleared. */
 int aug_enable_stage_timing(AugCtx *ctx, int on);

@@ -23,7 +23,7 @@ EXPORTS = ["aug_strerror", "aug_frame_count", "aug_workspace_bytes", "aug_valida
            "aug_create", "aug_destroy", "aug_last_status", "aug_rir_image_method",
            "aug_reverb_mix", "feat_stft_power", "feat_vtlp_logmel", "aug_pipeline",
            "aug_pipeline_host", "aug_enable_stage_timing", "aug_stage_times", "aug_launch_count",
-           "aug_measure_fp32_peak", "feat_vtlp_logmel_noalloc", "aug_last_host_bytes", "aug_upload_noise_bank", "aug_sample_params", "feat_mfcc", "feat_mean_var",
+           "aug_measure_fp32_peak", "feat_vtlp_logmel_noalloc", "aug_last_host_bytes", "aug_upload_noise_bank", "aug_hold_parking_slots", "aug_sample_params", "feat_mfcc", "feat_mean_var",
            "aug_bucket_by_length"]
 NOALLOC_MAX_BATCH = 256
 N_STAGES = 7
@@ -114,6 +114,8 @@ def lib() -> ctypes.CDLL:
         L.aug_bucket_by_length.argtypes = [vp, i32, i32, vp, vp]
         L.aug_sample_params.restype = i32
         L.aug_sample_params.argtypes = [ctypes.c_uint64, ctypes.POINTER(AugDist), i32, vp, vp]
+        L.aug_hold_parking_slots.restype = i32
+        L.aug_hold_parking_slots.argtypes = [vp, i32]
         L.aug_upload_noise_bank.restype = i32
         L.aug_upload_noise_bank.argtypes = [vp, vp, i64]
         L.aug_last_host_bytes.restype = i32
@@ -335,6 +337,9 @@ class AugContext:
                                             _ptr(table_dev), int(B), _ptr(feats_dev), int(T_max),
                                             _ptr(counts_dev), _ptr(wave_out_dev)),
                          "aug_pipeline", check)
+
+    def aug_hold_parking_slots(self, hold):
+        _check(lib().aug_hold_parking_slots(self._h, int(bool(hold))), "aug_hold_parking_slots")
 
     def aug_upload_noise_bank(self, bank_host, bank_len, check=True):
         return self._ret(lib().aug_upload_noise_bank(self._h, _ptr(bank_host), int(bank_len)),

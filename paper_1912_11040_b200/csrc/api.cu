@@ -78,7 +78,7 @@ int check_config(const AugConfig *c) {
 struct Layout {
     int n_part, route, n_bins, t_cap, nblk_cap;
     int64_t ws_stride;
-    int64_t off_xspec;
+    int64_t off_xspec, off_park, off_park_flags;
     int64_t off_tw, off_rir, off_hspec, off_ys, off_vv, off_energy, off_gain, off_melw, off_melstart,
         off_status, off_st_speech, off_st_bank, off_st_table, off_st_lengths,
         off_st_feats, off_st_counts, total;
@@ -100,6 +100,10 @@ Layout make_layout(const AugConfig &c) {
     l.off_hspec = take(sizeof(float2) * B * S * (l.route == aug::ROUTE_FUSED_8192 ? 2 : l.n_part) * aug::CONV_N2);
     l.nblk_cap = (c.max_samples + aug::CONV_BLK - 1) / aug::CONV_BLK;
     l.off_xspec = l.route == aug::ROUTE_STORED ? take(sizeof(float2) * B * S * l.nblk_cap * aug::CONV_N2) : -1;
+    // parking slots of the fused route, three per multiprocessor, when a row can have several noises
+    const bool parks = l.route == aug::ROUTE_FUSED_8192 && c.max_sources >= 3;
+    l.off_park = parks ? take(sizeof(float2) * (int64_t)aug::PARK_SMS * 3 * 2 * aug::CONV_N2) : -1;
+    l.off_park_flags = parks ? take(sizeof(int) * (int64_t)aug::PARK_SMS * 3) : -1;
     l.off_ys = take(sizeof(float) * B * l.ws_stride);
     l.off_vv = take(sizeof(float) * B * l.ws_stride);
     l.off_energy = take(sizeof(double) * 2 * B);
@@ -222,6 +226,9 @@ int aug_create(AugCtx **out, const AugConfig *cfg, void *cuda_stream) {
     ctx->hspec = reinterpret_cast<float2 *>(base + l.off_hspec);
     ctx->nblk_cap = l.nblk_cap;
     ctx->xspec = l.off_xspec >= 0 ? reinterpret_cast<float2 *>(base + l.off_xspec) : nullptr;
+    ctx->park = l.off_park >= 0 ? reinterpret_cast<float2 *>(base + l.off_park) : nullptr;
+    ctx->park_flags = l.off_park_flags >= 0 ? reinterpret_cast<int *>(base + l.off_park_flags) : nullptr;
+    ctx->n_sm = aug::PARK_SMS;
     ctx->ys = reinterpret_cast<float *>(base + l.off_ys);
     ctx->vv = reinterpret_cast<float *>(base + l.off_vv);
     ctx->energy = reinterpret_cast<double *>(base + l.off_energy);
@@ -260,6 +267,12 @@ int aug_create(AugCtx **out, const AugConfig *cfg, void *cuda_stream) {
         }
     }
     const int st0[2] = {-1, 0};
+    if (ctx->park_flags &&
+        cudaMemsetAsync(ctx->park_flags, 0, sizeof(int) * aug::PARK_SMS * 3, ctx->stream) != cudaSuccess) {
+        cudaFree(ctx->ws_base);
+        delete ctx;
+        return AUG_ECUDA;
+    }
     bool ok = cudaMemcpyAsync(ctx->tw, tw.data(), sizeof(float2) * augfft::TW_N,
                               cudaMemcpyHostToDevice, ctx->stream) == cudaSuccess &&
               cudaMemcpyAsync(ctx->status, st0, sizeof(st0), cudaMemcpyHostToDevice,
@@ -539,6 +552,18 @@ int aug_upload_noise_bank(AugCtx *ctx, const float *noise_bank_host, int64_t ban
                                 cudaMemcpyHostToDevice, ctx->stream));
     AUG_CUDA_OK(cudaStreamSynchronize(ctx->stream));
     ctx->bank_resident = bank_len;
+    return AUG_OK;
+}
+
+int aug_hold_parking_slots(AugCtx *ctx, int hold) {
+    if (!ctx) return AUG_EINVAL;
+    if (!ctx->park_flags) return AUG_OK;   // this context has no parking area
+    // all slots marked taken: every CTA then sums its noise sources in the time domain
+    std::vector<int> v((size_t)aug::PARK_SMS * 3, hold ? 1 : 0);
+    AUG_CUDA_OK(cudaStreamSynchronize(ctx->stream));
+    AUG_CUDA_OK(cudaMemcpyAsync(ctx->park_flags, v.data(), sizeof(int) * v.size(), cudaMemcpyHostToDevice,
+                                ctx->stream));
+    AUG_CUDA_OK(cudaStreamSynchronize(ctx->stream));
     return AUG_OK;
 }
 

@@ -14,6 +14,7 @@ constexpr int CONV_N2 = CONV_F / 2;     // complex FFT size
 #define AUG_FUSED16K_MIN_TAPS 0
 #endif
 constexpr int FUSED16K_MIN_TAPS = AUG_FUSED16K_MIN_TAPS;   // responses up to this length keep the 8192-point route
+constexpr int PARK_SMS = 160;       // multiprocessors that get parking slots (3 each) in the fused convolution
 constexpr int MAX_TAPS = 24576;
 constexpr int MAX_ORDER = 32;
 constexpr int MAX_HALF_W = 47;
@@ -61,6 +62,9 @@ struct AugCtx {
     float2 *hspec;         // [max_batch][max_sources][n_part][CONV_N2]
     float2 *xspec;         // [max_batch][max_sources][nblk_cap][CONV_N2]; NULL unless route == ROUTE_STORED
     int nblk_cap;          // blocks of an utterance of max_samples
+    float2 *park;          // [PARK_SMS * 3][8192] products of noise sources waiting for the last one; NULL if unused
+    int *park_flags;       // [PARK_SMS * 3] 1 = slot taken
+    int n_sm;              // multiprocessors with slots (PARK_SMS); CTAs on others sum in the time domain
     float *ys;             // [max_batch][ws_stride]
     float *vv;             // [max_batch][ws_stride]
     double *energy;        // [max_batch][2]

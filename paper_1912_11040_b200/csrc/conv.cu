@@ -11,7 +11,8 @@
 //                     nothing but y_s and v is stored.  The 8192-point complex
 //                     transform of the (even, odd) sample pairs runs as two
 //                     4096-point transforms joined by a radix-2 step (second half
-//                     of this file).  Noise sources are summed in the time domain.
+//                     of this file).  Several noise sources are summed in the frequency domain
+//                     through a small parking area in global memory (one inverse).
 //   longer            partitions of CONV_BLK = 4096 taps of an 8192-point transform,
 //                     Y_b = sum_p X_{b-p} H_p with X_j the spectrum of the 8192
 //                     samples that end with block j: block_spectra_kernel stores
@@ -685,16 +686,21 @@ rir_spectra2_kernel(const float *__restrict__ rir, const AugUttParams *__restric
     }
 }
 
+// PARK: rows may have several noise sources (the context allows three or more
+// sources); without it the kernel carries none of the parking code.
+template <bool PARK>
 __global__ void __launch_bounds__(CT, CONV_MINB)
 convolve_fused2_kernel(const float *__restrict__ speech, int64_t stride,
                        const int *__restrict__ lengths, const float *__restrict__ bank,
                        int64_t bank_len, const AugUttParams *__restrict__ table, int S_max,
                        const float2 *__restrict__ hspec, const float2 *__restrict__ tw,
                        float *__restrict__ ys, float *__restrict__ vv, int64_t ws_stride,
-                       double *__restrict__ energy, int *status, int n_cap, int ob) {
+                       double *__restrict__ energy, int *status, int n_cap, int ob,
+                       float2 *__restrict__ park, int *park_flags, int n_sm) {
     extern __shared__ __align__(16) float2 sm[];
     float2 *A = sm, *Bf = sm + SM_POINTS;
     __shared__ float red[CT / 32];
+    __shared__ int park_slot_s;
     const int b_first = blockIdx.x * CONV_RUN, utt = blockIdx.y, t = threadIdx.x;
     const int N = min(max(lengths[utt], 0), n_cap);
     if ((int64_t)b_first * ob >= N) return;
@@ -703,21 +709,45 @@ convolve_fused2_kernel(const float *__restrict__ speech, int64_t stride,
     if (n_src < 1 || n_src > S_max) n_src = 0;   // rejected row: silence (reported by step 1)
     const int m0 = (F2 - ob) / 4;            // first point of A and B that belongs to a block
 
-    // Noise sources are summed in the time domain (v is read back and added to for
-    // every source after the first); the energy is taken when the last one lands.
-    int last_noise = 0;
+    int last_noise = 0, n_noise = 0;
     for (int s = 1; s < n_src; ++s) {
         const float *x;
         int nlen;
-        if (source_of(row, s, nullptr, bank, bank_len, x, nlen)) last_noise = s;
-        else if (t == 0 && b_first == 0 && atomicCAS(&status[0], -1, utt) == -1) status[1] = aug::R_NOISE;
+        if (source_of(row, s, nullptr, bank, bank_len, x, nlen)) {
+            last_noise = s;
+            ++n_noise;
+        } else if (t == 0 && b_first == 0 && atomicCAS(&status[0], -1, utt) == -1) {
+            status[1] = aug::R_NOISE;
+        }
     }
+    // Several noise sources are summed in the frequency domain: the products of all
+    // but the last are parked in a 64 KB global slot (one per resident CTA of an SM,
+    // taken with a compare-and-swap; it stays in L2) and added to the last one's
+    // before the single inverse transform.  A CTA that finds no free slot -- more
+    // CTAs on the SM than slots -- sums in the time domain instead: v is read back
+    // and added to for every source after the first, one inverse transform each.
+    int park_slot = -1;
+    if (PARK && n_noise > 1 && park != nullptr) {
+        if (t == 0) {
+            unsigned smid;
+            asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+            int got = -1;
+            if ((int)smid < n_sm) {
+                for (int i = 0; i < CONV_MINB && got < 0; ++i)
+                    if (atomicCAS(&park_flags[smid * CONV_MINB + i], 0, 1) == 0) got = smid * CONV_MINB + i;
+            }
+            park_slot_s = got;
+        }
+        __syncthreads();
+        park_slot = park_slot_s;
+    }
+    float2 *slot = park_slot >= 0 ? park + (int64_t)park_slot * (4 * NQ2 * CT) : nullptr;
     // A CTA works through CONV_RUN consecutive blocks: while it loads the segment of
     // block b it asks for the new samples of block b + 1 to be brought into L2.
     for (int b = b_first; b < b_first + CONV_RUN && (int64_t)b * ob < N; ++b) {
     const int n_left = min(N - b * ob, ob);
     const bool more = b + 1 < b_first + CONV_RUN;
-    bool v_written = false;
+    bool v_written = false, v_parked = false;
     for (int s = 0; s < n_src; ++s) {
         const float *x;
         int nlen;
@@ -729,9 +759,15 @@ convolve_fused2_kernel(const float *__restrict__ speech, int64_t stride,
             fft2x4096_from_regs(va, vb, A, Bf, t, tw);
         }
         const float2 *H = hspec + ((int64_t)utt * S_max + s) * NB2;
+        // what happens to this source's products: inverse-transformed right away (0),
+        // parked for a later noise source (1: first one, 2: added to what is parked),
+        // or joined by the parked sum before the inverse (3)
+        int mode = 0;
+        if (PARK && s != 0 && slot != nullptr) mode = s == last_noise ? 3 : (v_parked ? 2 : 1);
 #pragma unroll 2
         for (int q = 0; q < NQ2; ++q) {
             const int k = t + CT * q;
+            float2 *pk = slot + (4 * q) * CT + t;      // this thread's four parked products, CT apart
             if (k == 0) {
                 const float2 uh = __ldg(&tw[tw_index(F2, N2 / 2)]);
                 Edge x4 = edge_forward(A[pad0(0)], Bf[pad0(0)], A[pad0(N2 / 2)], Bf[pad0(N2 / 2)], uh);
@@ -740,7 +776,20 @@ convolve_fused2_kernel(const float *__restrict__ speech, int64_t stride,
                 x4.mid = cmul(x4.mid, __ldg(&H[N2]));
                 x4.q1 = cmul(x4.q1, __ldg(&H[N2 / 2]));
                 x4.q3 = cmul(x4.q3, __ldg(&H[N2 + N2 / 2]));
-                edge_inverse(x4, uh, A[pad0(0)], Bf[pad0(0)], A[pad0(N2 / 2)], Bf[pad0(N2 / 2)]);
+                if (PARK && mode >= 2) {
+                    x4.dc = cadd(x4.dc, pk[0]);
+                    x4.mid = cadd(x4.mid, pk[CT]);
+                    x4.q1 = cadd(x4.q1, pk[2 * CT]);
+                    x4.q3 = cadd(x4.q3, pk[3 * CT]);
+                }
+                if (PARK && (mode == 1 || mode == 2)) {
+                    pk[0] = x4.dc;
+                    pk[CT] = x4.mid;
+                    pk[2 * CT] = x4.q1;
+                    pk[3 * CT] = x4.q3;
+                } else {
+                    edge_inverse(x4, uh, A[pad0(0)], Bf[pad0(0)], A[pad0(N2 / 2)], Bf[pad0(N2 / 2)]);
+                }
             } else {
                 const float2 w = __ldg(&tw[tw_index(NB2, k)]), u = __ldg(&tw[tw_index(F2, k)]);
                 Quad x4 = quad_forward(A[pad0(k)], A[pad0(N2 - k)], Bf[pad0(k)], Bf[pad0(N2 - k)], w, u);
@@ -748,8 +797,27 @@ convolve_fused2_kernel(const float *__restrict__ speech, int64_t stride,
                 x4.nk = cmul(x4.nk, __ldg(&H[NB2 - k]));
                 x4.mk = cmul(x4.mk, __ldg(&H[N2 - k]));
                 x4.pk = cmul(x4.pk, __ldg(&H[N2 + k]));
-                quad_inverse(x4, w, u, A[pad0(k)], A[pad0(N2 - k)], Bf[pad0(k)], Bf[pad0(N2 - k)]);
+                if (PARK && mode >= 2) {
+                    x4.k = cadd(x4.k, pk[0]);
+                    x4.nk = cadd(x4.nk, pk[CT]);
+                    x4.mk = cadd(x4.mk, pk[2 * CT]);
+                    x4.pk = cadd(x4.pk, pk[3 * CT]);
+                }
+                if (PARK && (mode == 1 || mode == 2)) {
+                    pk[0] = x4.k;
+                    pk[CT] = x4.nk;
+                    pk[2 * CT] = x4.mk;
+                    pk[3 * CT] = x4.pk;
+                } else {
+                    quad_inverse(x4, w, u, A[pad0(k)], A[pad0(N2 - k)], Bf[pad0(k)], Bf[pad0(N2 - k)]);
+                }
             }
+        }
+        if (PARK && (mode == 1 || mode == 2)) {
+            // every thread reads back only what it parked itself: no fence is needed
+            v_parked = true;
+            __syncthreads();   // the buffers are refilled by the next source
+            continue;
         }
         __syncthreads();
         fft2x4096_in_place(A, Bf, t, tw);
@@ -801,6 +869,10 @@ convolve_fused2_kernel(const float *__restrict__ speech, int64_t stride,
         for (int i = t; i < n_left; i += CT) dst[i] = 0.f;
     }
     }   // blocks of the run
+    if (PARK && park_slot >= 0) {
+        __syncthreads();                                  // all reads of the slot are done
+        if (t == 0) atomicExch(&park_flags[park_slot], 0);
+    }
 }
 
 constexpr size_t FFT_SMEM = sizeof(float2) * SM_POINTS;
@@ -854,15 +926,16 @@ int launch_convolve_finish(AugCtx *ctx, const float *speech, int64_t stride, con
     const int nblk = (max_len + BLK - 1) / BLK;
     dim3 grid(nblk, B);
     if (ctx->route == aug::ROUTE_FUSED_8192) {
-        AUG_CUDA_OK(cudaFuncSetAttribute(convolve_fused2_kernel,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FFT2_SMEM));
         // every block yields the F2 - (taps - 1) outputs that see no wrap-around, cut to a multiple of 4
         const int ob = (F2 - c.rir_taps + 1) & ~3;
         const int nblk2 = (max_len + ob - 1) / ob;
         dim3 grid2((nblk2 + CONV_RUN - 1) / CONV_RUN, B);
-        convolve_fused2_kernel<<<grid2, CT, FFT2_SMEM, ctx->stream>>>(
+        auto kern = ctx->park ? convolve_fused2_kernel<true> : convolve_fused2_kernel<false>;
+        AUG_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FFT2_SMEM));
+        kern<<<grid2, CT, FFT2_SMEM, ctx->stream>>>(
             speech, stride, lengths, bank, bank_len, table, c.max_sources, ctx->hspec, ctx->tw,
-            ctx->ys, ctx->vv, ctx->ws_stride, ctx->energy, ctx->status, max_len, ob);
+            ctx->ys, ctx->vv, ctx->ws_stride, ctx->energy, ctx->status, max_len, ob, ctx->park,
+            ctx->park_flags, ctx->n_sm);
     } else if (!stored_route(ctx)) {
         convolve_fused_kernel<<<grid, CT, FFT_SMEM, ctx->stream>>>(
             speech, stride, lengths, bank, bank_len, table, c.max_sources, ctx->n_part, ctx->hspec,

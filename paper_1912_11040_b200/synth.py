@@ -258,7 +258,9 @@ def make_workload(index: int, seed: int = 0, *, batch: Optional[int] = None,
                          t60=r["t60"], order=ordr, n_noise=r["n_noise"], snr=r["snr"],
                          alpha=r["alpha"], noise_align=noise_align)
     cfg = dict(_COMMON)
+    # the context is sized for what the workload holds: speech plus its largest noise count
     cfg.update(n_mel=r["n_mel"], n_fft=r["n_fft"], max_order=ordr,
-               rir_taps=r["taps"] if taps is None else int(taps))
+               rir_taps=r["taps"] if taps is None else int(taps),
+               max_sources=1 + int(r["n_noise"][1]))
     return Workload(name=f"config{index}", cfg=cfg, lengths=lengths, speech=speech,
                     bank=bank, table=table)

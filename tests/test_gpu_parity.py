@@ -152,6 +152,36 @@ def test_pipeline_with_unaligned_and_very_short_noise_stretches(index):
     check_pipeline_against_oracle(dev, F, counts, wave, oracle_batch(w))
 
 
+def test_fused_route_sums_three_noise_sources():
+    """8192 taps, rows with one, two and three noise sources: the products of all but the
+    last noise wait in the parking slot and are added before the single inverse transform."""
+    w = small(2, batch=3, dur_scale=0.15)
+    w.cfg["max_sources"] = 4
+    rng = np.random.default_rng(5)
+    for b, n_src in enumerate((2, 3, 4)):
+        row = w.table[b]
+        row["n_src"] = n_src
+        for s in range(1, n_src):
+            row["src_pos"][s] = [rng.uniform(0.4, float(row["room"][a]) - 0.4) for a in range(3)]
+            row["noise_len"][s - 1] = 4000 + 1236 * s
+            row["noise_offset"][s - 1] = 2000 * s + 4 * b
+            row["noise_weight"][s - 1] = 0.4 + 0.3 * s
+    dev = Device(w)
+    assert binding.aug_validate_params(dev.cfg, w.table, w.bank.size) == (0, -1)
+    F, counts, wave = dev.pipeline(want_wave=True)
+    assert dev.ctx.aug_last_status() == (-1, 0)
+    check_pipeline_against_oracle(dev, F, counts, wave, oracle_batch(w))
+    # a second call finds the slots free again and gives the same answer
+    F2, counts2, wave2 = dev.pipeline(want_wave=True)
+    orc = oracle_batch(w)
+    check_pipeline_against_oracle(dev, F2, counts2, wave2, orc)
+    # with every slot held the sources are summed in the time domain: same answer again
+    dev.ctx.aug_hold_parking_slots(True)
+    F3, counts3, wave3 = dev.pipeline(want_wave=True)
+    check_pipeline_against_oracle(dev, F3, counts3, wave3, orc)
+    dev.ctx.aug_hold_parking_slots(False)
+
+
 def test_pipeline_edge_lengths_and_no_noise():
     w = small(2, batch=8, dur_scale=0.12)
     w.lengths[:6] = [0, 1, 399, 400, 559, 560]
@@ -280,6 +310,7 @@ def test_pipeline_runs_on_a_table_from_the_library_sampler():
     d.snr_lo, d.snr_hi, d.alpha_lo, d.alpha_hi = 0, 30, 0.8, 1.2
     d.wall_margin, d.min_src_mic_dist, d.min_noise_len, d.bank_len = 0.3, 0.5, 4000, w.bank.size
     _, w.table = binding.aug_sample_params(123, d, w.lengths)
+    w.cfg["max_sources"] = 4           # up to three noise sources per row
     dev = Device(w)
     assert binding.aug_validate_params(dev.cfg, w.table, w.bank.size) == (0, -1)
     F, counts, wave = dev.pipeline(want_wave=True)
@@ -335,6 +366,7 @@ def test_pipeline_at_the_configuration_limits():
     count a context accepts, on one short utterance."""
     w = small(5, batch=1, dur_scale=1.0 / 60.0, taps=24576, order=32)     # 1 s, 1024-point FFT, 128 mel
     w.cfg["frac_half_width"] = 47
+    w.cfg["max_sources"] = 4
     row = w.table[0]
     rng = np.random.default_rng(9)
     row["n_src"] = 4
