@@ -187,7 +187,8 @@ __host__ __device__ constexpr int fbuf_floats(int FT, int M) {
 #define FEAT_MINB 3           // CTAs per SM the register budget is set for
 #endif
 // MODE 0: wave -> power (global).  MODE 1: y_s + g v -> features.
-template <int K, int MODE>
+// TILES: consecutive tiles one CTA works through.
+template <int K, int MODE, int TILES>
 __global__ void __launch_bounds__(FEAT_THREADS, FEAT_MINB)
 frames_kernel(const float *__restrict__ in_a, const float *__restrict__ in_b, int64_t in_stride,
               const float *__restrict__ gain, const AugUttParams *__restrict__ table,
@@ -195,7 +196,7 @@ frames_kernel(const float *__restrict__ in_a, const float *__restrict__ in_b, in
               const aug::MelBin *__restrict__ melw, const int *__restrict__ melstart,
               const float2 *__restrict__ tw, float floor_v, float pad_v, int comp,
               float *__restrict__ out, int *__restrict__ counts, int n_cap) {
-    constexpr int E = Plan<K>::E, FT = Plan<K>::FT, TILES = Plan<K>::TILES, NBP = K / 2 + 1;
+    constexpr int E = Plan<K>::E, FT = Plan<K>::FT, NBP = K / 2 + 1;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float2 *fbuf = reinterpret_cast<float2 *>(smem_raw);            // [NGROUP][K + K/8]; later the interval sums
     float *ptile = reinterpret_cast<float *>(smem_raw) + fbuf_floats<K>(FT, M);    // [FT][NBP]
@@ -367,11 +368,16 @@ int launch_frames(AugCtx *ctx, const float *a, const float *b, int64_t stride, c
                         sizeof(float) * chunk_cap + sizeof(aug::MelBin) * (NBP + 1) +
                         sizeof(int) * (c.n_mel + 2);
     if (smem > 227 * 1024) return AUG_ECAP;
-    AUG_CUDA_OK(cudaFuncSetAttribute(frames_kernel<K, MODE>,
-                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    constexpr int RUN = FT * Plan<K>::TILES;
+    // A CTA works through a run of tiles (window values, filterbank tables and other
+    // set-up once per run) unless the batch is so small that single tiles are needed
+    // to give every multiprocessor something to do.
+    const int n_tiles = (T_max + FT - 1) / FT;
+    const bool runs = (int64_t)n_tiles * B >= 2 * 148 * Plan<K>::TILES;
+    const int RUN = FT * (runs ? Plan<K>::TILES : 1);
     dim3 grid((T_max + RUN - 1) / RUN, B);
-    frames_kernel<K, MODE><<<grid, FEAT_THREADS, smem, ctx->stream>>>(
+    auto kern = runs ? frames_kernel<K, MODE, Plan<K>::TILES> : frames_kernel<K, MODE, 1>;
+    AUG_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    kern<<<grid, FEAT_THREADS, smem, ctx->stream>>>(
         a, b, stride, ctx->gain, table, lengths, c.win, c.hop, c.n_mel, T_max, ctx->melw,
         ctx->melstart, ctx->tw, c.log_floor, c.pad_value, c.compression, out, counts,
         (int)(stride < 0x7fffffff ? stride : 0x7fffffff));
