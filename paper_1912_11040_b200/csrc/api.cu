@@ -87,8 +87,7 @@ struct Layout {
 Layout make_layout(const AugConfig &c) {
     Layout l;
     l.n_part = (c.rir_taps + aug::CONV_BLK - 1) / aug::CONV_BLK;
-    l.route = c.rir_taps <= aug::FUSED16K_MIN_TAPS ? aug::ROUTE_FUSED_4096
-              : l.n_part <= 2 ? aug::ROUTE_FUSED_8192 : aug::ROUTE_STORED;
+    l.route = l.n_part <= 2 ? aug::ROUTE_FUSED_8192 : aug::ROUTE_STORED;
     l.n_bins = c.n_fft / 2 + 1;
     l.t_cap = aug_frame_count(c.max_samples, c.win, c.hop);
     l.ws_stride = align_up(c.max_samples, 4);

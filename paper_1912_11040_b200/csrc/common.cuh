@@ -10,10 +10,6 @@ namespace aug {
 constexpr int CONV_BLK = 4096;          // output samples per convolution block
 constexpr int CONV_F = 2 * CONV_BLK;    // real FFT size of one block
 constexpr int CONV_N2 = CONV_F / 2;     // complex FFT size
-#ifndef AUG_FUSED16K_MIN_TAPS
-#define AUG_FUSED16K_MIN_TAPS 0
-#endif
-constexpr int FUSED16K_MIN_TAPS = AUG_FUSED16K_MIN_TAPS;   // responses up to this length keep the 8192-point route
 constexpr int PARK_SMS = 160;       // multiprocessors that get parking slots (3 each) in the fused convolution
 constexpr int MAX_TAPS = 24576;
 constexpr int MAX_ORDER = 32;
@@ -27,12 +23,10 @@ constexpr int EV_RING = 256;
 constexpr int HOST_CHUNKS = AUG_HOST_CHUNKS;   // pipeline depth of aug_pipeline_host
 
 // How step 2 is run, fixed by the response length at aug_create:
-//   ROUTE_FUSED_4096  rir_taps <= FUSED16K_MIN_TAPS: one partition of an 8192-point transform
-//                     (4096 outputs per block), one kernel
 //   ROUTE_FUSED_8192  rir_taps <= 8192: one partition of a 16384-point transform
 //                     (16384 - taps + 1 outputs per block), one kernel
 //   ROUTE_STORED      longer: partitions of 4096 taps, block spectra stored once and reused
-enum Route { ROUTE_FUSED_4096 = 0, ROUTE_FUSED_8192 = 1, ROUTE_STORED = 2 };
+enum Route { ROUTE_FUSED_8192 = 1, ROUTE_STORED = 2 };
 
 enum Reason { R_NONE = 0, R_NSRC = 1, R_ORDER = 2, R_NOISE = 3 };
 

@@ -20,8 +20,6 @@
 //                     block needs (mostly from L2), multiply-accumulates in registers
 //                     and inverse-transforms.  Noise sources are summed in the
 //                     frequency domain: two inverse transforms per block.
-//   (convolve_fused_kernel, one partition of the 8192-point transform, is kept
-//   behind the compile-time knob AUG_FUSED16K_MIN_TAPS.)
 //
 // A real transform of F points is a complex transform of F/2 points on (even, odd)
 // sample pairs followed by the usual split; in the 8192-point routes thread t owns
@@ -40,9 +38,6 @@ constexpr int CT = 256;               // threads per CTA
 constexpr int E = N2 / CT;            // 16 points per thread: three radix-16 passes
 constexpr int NQ = N2 / 2 / CT;       // 8 bin pairs per thread
 constexpr int SM_POINTS = padded_points(N2);
-#ifndef CONV_RUN
-#define CONV_RUN 1                   // consecutive 16384-point blocks one CTA works through
-#endif
 #ifndef CONV_MINB
 #define CONV_MINB 3                  // CTAs per SM the register budget is set for
 #endif
@@ -256,61 +251,6 @@ rir_spectra_kernel(const float *__restrict__ rir, const AugUttParams *__restrict
         spectrum_pair(sm, tw, k, a, b);
         out[slot_a(k)] = make_float2(a.x * scale, a.y * scale);
         out[slot_b(k)] = make_float2(b.x * scale, b.y * scale);
-    }
-}
-
-// ---------------------------------------------------------------- one partition: fused
-__global__ void __launch_bounds__(CT, CONV_MINB)
-convolve_fused_kernel(const float *__restrict__ speech, int64_t stride,
-                      const int *__restrict__ lengths, const float *__restrict__ bank,
-                      int64_t bank_len, const AugUttParams *__restrict__ table, int S_max, int P,
-                      const float2 *__restrict__ hspec, const float2 *__restrict__ tw,
-                      float *__restrict__ ys, float *__restrict__ vv, int64_t ws_stride,
-                      double *__restrict__ energy, int *status, int n_cap) {
-    extern __shared__ __align__(16) float2 sm[];
-    __shared__ float red[CT / 32];
-    const int b = blockIdx.x, utt = blockIdx.y, t = threadIdx.x;
-    const int N = min(max(lengths[utt], 0), n_cap);
-    if ((int64_t)b * BLK >= N) return;
-    const AugUttParams &row = table[utt];
-    int n_src = row.n_src;
-    if (n_src < 1 || n_src > S_max) n_src = 0;   // rejected row: silence (reported by step 1)
-    const int n_out = n_src > 1 ? 2 : (n_src == 1 ? 1 : 0);
-
-    for (int o = 0; o < n_out; ++o) {
-        float2 acc[NQ][2];
-#pragma unroll
-        for (int q = 0; q < NQ; ++q) acc[q][0] = acc[q][1] = make_float2(0.f, 0.f);
-        const int s_lo = o ? 1 : 0, s_hi = o ? n_src : 1;
-        for (int s = s_lo; s < s_hi; ++s) {
-            const float *x;
-            int nlen;
-            if (!source_of(row, s, speech + (int64_t)utt * stride, bank, bank_len, x, nlen)) {
-                if (t == 0 && b == 0 && atomicCAS(&status[0], -1, utt) == -1) status[1] = aug::R_NOISE;
-                continue;
-            }
-            for (int p = 0; p < P && p <= b; ++p) {
-                float2 v[1][E];
-                load_segment(v, x, s != 0, nlen, (b - p - 1) * BLK, N, t);
-                fft4096_from_regs(v, sm, t, tw);
-                const float2 *H = hspec + (((int64_t)utt * S_max + s) * P + p) * N2;
-#pragma unroll
-                for (int q = 0; q < NQ; ++q) {
-                    const int k = t + CT * q;
-                    float2 xa, xb;
-                    spectrum_pair(sm, tw, k, xa, xb);
-                    mac_pair(acc[q][0], acc[q][1], xa, xb, __ldg(&H[slot_a(k)]), __ldg(&H[slot_b(k)]), k);
-                }
-                __syncthreads();   // sm is overwritten by the next transform
-            }
-        }
-        float *dst = (o ? vv : ys) + (int64_t)utt * ws_stride + (int64_t)b * BLK;
-        finish_block(acc, sm, tw, t, dst, N - b * BLK, &energy[2 * utt + o], red);
-    }
-    if (n_src <= 1) {
-        // no noise: v is defined as silence
-        float *dst = vv + (int64_t)utt * ws_stride + (int64_t)b * BLK;
-        for (int i = t; i < BLK && b * BLK + i < N; i += CT) dst[i] = 0.f;
     }
 }
 
@@ -534,19 +474,6 @@ __device__ __noinline__ void fft2x4096_tail(float2 *A, float2 *B, int t, const f
     __syncthreads();
 }
 
-// Ask for samples [start, start + count) of a source, cut to [0, N), to be brought
-// into L2: one 128-byte line per thread and step.  A looped source maps the sample
-// index into its stretch.
-__device__ __forceinline__ void prefetch_l2(const float *x, bool looped, int nlen, int start, int count,
-                                            int N, int t) {
-    const int end = min(start + count, N);
-    for (int i = start + 32 * t; i < end; i += 32 * CT) {
-        if (i < 0) continue;
-        const float *p = x + (looped ? i % nlen : i);
-        asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
-    }
-}
-
 // Both half transforms of a segment held in registers; on return A and B hold the
 // 4096-point transforms of the even and odd pairs, complete and synchronised.
 __device__ __forceinline__ void fft2x4096_from_regs(float2 (*va)[E], float2 (*vb)[E], float2 *A,
@@ -701,9 +628,9 @@ convolve_fused2_kernel(const float *__restrict__ speech, int64_t stride,
     float2 *A = sm, *Bf = sm + SM_POINTS;
     __shared__ float red[CT / 32];
     __shared__ int park_slot_s;
-    const int b_first = blockIdx.x * CONV_RUN, utt = blockIdx.y, t = threadIdx.x;
+    const int b = blockIdx.x, utt = blockIdx.y, t = threadIdx.x;
     const int N = min(max(lengths[utt], 0), n_cap);
-    if ((int64_t)b_first * ob >= N) return;
+    if ((int64_t)b * ob >= N) return;
     const AugUttParams &row = table[utt];
     int n_src = row.n_src;
     if (n_src < 1 || n_src > S_max) n_src = 0;   // rejected row: silence (reported by step 1)
@@ -716,7 +643,7 @@ convolve_fused2_kernel(const float *__restrict__ speech, int64_t stride,
         if (source_of(row, s, nullptr, bank, bank_len, x, nlen)) {
             last_noise = s;
             ++n_noise;
-        } else if (t == 0 && b_first == 0 && atomicCAS(&status[0], -1, utt) == -1) {
+        } else if (t == 0 && b == 0 && atomicCAS(&status[0], -1, utt) == -1) {
             status[1] = aug::R_NOISE;
         }
     }
@@ -742,11 +669,7 @@ convolve_fused2_kernel(const float *__restrict__ speech, int64_t stride,
         park_slot = park_slot_s;
     }
     float2 *slot = park_slot >= 0 ? park + (int64_t)park_slot * (4 * NQ2 * CT) : nullptr;
-    // A CTA works through CONV_RUN consecutive blocks: while it loads the segment of
-    // block b it asks for the new samples of block b + 1 to be brought into L2.
-    for (int b = b_first; b < b_first + CONV_RUN && (int64_t)b * ob < N; ++b) {
     const int n_left = min(N - b * ob, ob);
-    const bool more = b + 1 < b_first + CONV_RUN;
     bool v_written = false, v_parked = false;
     for (int s = 0; s < n_src; ++s) {
         const float *x;
@@ -755,7 +678,6 @@ convolve_fused2_kernel(const float *__restrict__ speech, int64_t stride,
         {
             float2 va[1][E], vb[1][E];
             load_segment4(va, vb, x, s != 0, nlen, (b + 1) * ob - F2, N, t);
-            if (more) prefetch_l2(x, s != 0, nlen, (b + 1) * ob, ob, N, t);
             fft2x4096_from_regs(va, vb, A, Bf, t, tw);
         }
         const float2 *H = hspec + ((int64_t)utt * S_max + s) * NB2;
@@ -868,7 +790,6 @@ convolve_fused2_kernel(const float *__restrict__ speech, int64_t stride,
         float *dst = vv + (int64_t)utt * ws_stride + (int64_t)b * ob;
         for (int i = t; i < n_left; i += CT) dst[i] = 0.f;
     }
-    }   // blocks of the run
     if (PARK && park_slot >= 0) {
         __syncthreads();                                  // all reads of the slot are done
         if (t == 0) atomicExch(&park_flags[park_slot], 0);
@@ -929,17 +850,13 @@ int launch_convolve_finish(AugCtx *ctx, const float *speech, int64_t stride, con
         // every block yields the F2 - (taps - 1) outputs that see no wrap-around, cut to a multiple of 4
         const int ob = (F2 - c.rir_taps + 1) & ~3;
         const int nblk2 = (max_len + ob - 1) / ob;
-        dim3 grid2((nblk2 + CONV_RUN - 1) / CONV_RUN, B);
+        dim3 grid2(nblk2, B);
         auto kern = ctx->park ? convolve_fused2_kernel<true> : convolve_fused2_kernel<false>;
         AUG_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FFT2_SMEM));
         kern<<<grid2, CT, FFT2_SMEM, ctx->stream>>>(
             speech, stride, lengths, bank, bank_len, table, c.max_sources, ctx->hspec, ctx->tw,
             ctx->ys, ctx->vv, ctx->ws_stride, ctx->energy, ctx->status, max_len, ob, ctx->park,
             ctx->park_flags, ctx->n_sm);
-    } else if (!stored_route(ctx)) {
-        convolve_fused_kernel<<<grid, CT, FFT_SMEM, ctx->stream>>>(
-            speech, stride, lengths, bank, bank_len, table, c.max_sources, ctx->n_part, ctx->hspec,
-            ctx->tw, ctx->ys, ctx->vv, ctx->ws_stride, ctx->energy, ctx->status, max_len);
     } else {
         spectral_convolve_kernel<<<grid, CT, FFT_SMEM, ctx->stream>>>(
             lengths, bank, bank_len, table, c.max_sources, ctx->n_part, ctx->hspec, ctx->xspec,
