@@ -182,6 +182,31 @@ def test_fused_route_sums_three_noise_sources():
     dev.ctx.aug_hold_parking_slots(False)
 
 
+@pytest.mark.parametrize("n_fft,win,hop", [(512, 512, 200), (512, 400, 125), (1024, 800, 200)])
+def test_pipeline_with_other_window_and_hop(n_fft, win, hop):
+    """Window and hop are configuration fields: a window as long as the transform with a
+    stretch per tile that needs a second round of staging loads, a hop that is not a
+    multiple of four samples (scalar staging), and the 50 ms window of the paper's
+    Section 3 on the 1024-point transform."""
+    w = small(1, batch=3, dur_scale=0.8)
+    w.cfg.update(n_fft=n_fft, win=win, hop=hop)
+    w.lengths[1] = win + 5 * hop + 3
+    w.lengths[2] = win - 1
+    dev = Device(w)
+    F, counts, wave = dev.pipeline(want_wave=True)
+    assert dev.ctx.aug_last_status() == (-1, 0)
+    check_pipeline_against_oracle(dev, F, counts, wave, oracle_batch(w))
+    assert list(counts.cpu().numpy()[1:]) == [6, 0]
+    # steps 3 and 4 on their own, same settings
+    P, c2 = dev.stft_power(dev.speech)
+    for b in range(w.B):
+        x = w.speech[b, : w.lengths[b]].astype(np.float64)
+        ref = oracle.stft_power(x, win, hop, n_fft)
+        assert int(c2[b]) == ref.shape[0]
+        if ref.shape[0]:
+            assert np.max(np.abs(P[b, : ref.shape[0]].cpu().numpy() - ref)) <= 2e-6 * ref.max()
+
+
 def test_pipeline_edge_lengths_and_no_noise():
     w = small(2, batch=8, dur_scale=0.12)
     w.lengths[:6] = [0, 1, 399, 400, 559, 560]
