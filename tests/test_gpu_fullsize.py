@@ -20,9 +20,11 @@ def _sample(w, k):
     return sorted(set(picks))[:k]
 
 
-@pytest.mark.parametrize("index,n_check", [(1, 3), (2, 3), (3, 2), (4, 3), (5, 1)])
-def test_full_size_workload(index, n_check):
-    w = synth.make_workload(index, seed=0)
+# (the last case draws noise stretches at any offset and of any length: scalar loads)
+@pytest.mark.parametrize("index,n_check,noise_align",
+                         [(1, 3, 4), (2, 3, 4), (3, 2, 4), (4, 3, 4), (5, 1, 4), (4, 2, 1)])
+def test_full_size_workload(index, n_check, noise_align):
+    w = synth.make_workload(index, seed=0, noise_align=noise_align)
     dev = Device(w)
     rc, bad = binding.aug_validate_params(dev.cfg, w.table, w.bank.size)
     assert rc == 0, bad
