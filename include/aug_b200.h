@@ -178,7 +178,12 @@ int aug_last_status(AugCtx *ctx, int *utt_host, int *reason_host);
  * For each source the sum runs over the image lattice |kx|+|ky|+|kz| <= order
  * (or the cube, see AugLattice);
  * an image at distance d adds (prod beta^hits / d) times a Hann-windowed sinc
- * (half width frac_half_width) centred at d*fs/sound_speed samples. */
+ * (half width frac_half_width) centred at d*fs/sound_speed samples.
+ * Microphone arrays (the two microphones 6.8 cm apart of the far-field experiment
+ * in Section 4): a row describes ONE microphone.  For C channels the caller passes
+ * C rows per utterance -- row C*u + c is channel c of utterance u -- that differ
+ * only in `mic`, with the speech row and length repeated, and reads channel c from
+ * row C*u + c of every output.  Each row is mixed at the row's snr_db on its own. */
 int aug_rir_image_method(AugCtx *ctx, const AugUttParams *table_dev, int B, float *rir_dev);
 
 /* -------------------------------------------------------------- step 2

@@ -207,6 +207,12 @@ int aug_create(AugCtx **out, const AugConfig *cfg, void *cuda_stream) {
         delete ctx;
         return AUG_ECUDA;
     }
+    if (cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&ctx->smem_per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor,
+                               ctx->device) != cudaSuccess) {
+        delete ctx;
+        return AUG_ECUDA;
+    }
     const Layout l = make_layout(*cfg);
     ctx->n_part = l.n_part;
     ctx->route = l.route;

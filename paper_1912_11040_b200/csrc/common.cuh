@@ -3,6 +3,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "../../include/aug_b200.h"
 
 namespace aug {
@@ -43,6 +45,8 @@ struct AugCtx {
     AugConfig cfg;
     cudaStream_t stream;
     int device;
+    int sm_count;          // multiprocessors of the device
+    int smem_per_sm;       // shared memory of one multiprocessor, bytes
     int n_part;            // RIR partitions of CONV_BLK taps
     int route;             // aug::Route
     int n_bins;            // n_fft/2 + 1
@@ -89,6 +93,25 @@ struct AugCtx {
         cudaError_t e__ = (expr);                 \
         if (e__ != cudaSuccess) return AUG_ECUDA; \
     } while (0)
+
+// Let kernel Kern use as much dynamic shared memory as the device allows (the
+// opt-in limit less the kernel's static shared memory).  The attribute belongs to
+// the device's copy of the kernel, not to a context, so it is set once per device
+// and to the largest value any configuration can ask for.
+template <auto Kern>
+inline int smem_opt_in(int device) {
+    static std::atomic<unsigned long long> done{0};
+    const unsigned long long bit = 1ull << (device & 63);
+    if (done.load(std::memory_order_acquire) & bit) return AUG_OK;
+    int optin = 0;
+    cudaFuncAttributes fa;
+    AUG_CUDA_OK(cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device));
+    AUG_CUDA_OK(cudaFuncGetAttributes(&fa, Kern));
+    AUG_CUDA_OK(cudaFuncSetAttribute(Kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     optin - (int)fa.sharedSizeBytes));
+    done.fetch_or(bit, std::memory_order_release);
+    return AUG_OK;
+}
 
 // Launchers (defined next to their kernels).  They enqueue on ctx->stream unless a
 // stream is passed.

@@ -805,8 +805,7 @@ int launch_rir_spectra(AugCtx *ctx, const float *rir, const AugUttParams *table,
                        cudaStream_t st) {
     const AugConfig &c = ctx->cfg;
     if (ctx->route == aug::ROUTE_FUSED_8192) {
-        AUG_CUDA_OK(cudaFuncSetAttribute(rir_spectra2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)FFT2_SMEM));
+        if (smem_opt_in<rir_spectra2_kernel>(ctx->device) != AUG_OK) return AUG_ECUDA;
         dim3 grid(c.max_sources, B);
         rir_spectra2_kernel<<<grid, CT, FFT2_SMEM, st>>>(rir, table, c.max_sources, c.rir_taps, ctx->tw,
                                                          ctx->hspec);
@@ -852,7 +851,9 @@ int launch_convolve_finish(AugCtx *ctx, const float *speech, int64_t stride, con
         const int nblk2 = (max_len + ob - 1) / ob;
         dim3 grid2(nblk2, B);
         auto kern = ctx->park ? convolve_fused2_kernel<true> : convolve_fused2_kernel<false>;
-        AUG_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FFT2_SMEM));
+        if ((ctx->park ? smem_opt_in<convolve_fused2_kernel<true>>(ctx->device)
+                       : smem_opt_in<convolve_fused2_kernel<false>>(ctx->device)) != AUG_OK)
+            return AUG_ECUDA;
         kern<<<grid2, CT, FFT2_SMEM, ctx->stream>>>(
             speech, stride, lengths, bank, bank_len, table, c.max_sources, ctx->hspec, ctx->tw,
             ctx->ys, ctx->vv, ctx->ws_stride, ctx->energy, ctx->status, max_len, ob, ctx->park,

@@ -372,11 +372,13 @@ int launch_frames(AugCtx *ctx, const float *a, const float *b, int64_t stride, c
     // set-up once per run) unless the batch is so small that single tiles are needed
     // to give every multiprocessor something to do.
     const int n_tiles = (T_max + FT - 1) / FT;
-    const bool runs = (int64_t)n_tiles * B >= 2 * 148 * Plan<K>::TILES;
+    const bool runs = (int64_t)n_tiles * B >= 2 * (int64_t)ctx->sm_count * Plan<K>::TILES;
     const int RUN = FT * (runs ? Plan<K>::TILES : 1);
     dim3 grid((T_max + RUN - 1) / RUN, B);
     auto kern = runs ? frames_kernel<K, MODE, Plan<K>::TILES> : frames_kernel<K, MODE, 1>;
-    AUG_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    if ((runs ? smem_opt_in<frames_kernel<K, MODE, Plan<K>::TILES>>(ctx->device)
+              : smem_opt_in<frames_kernel<K, MODE, 1>>(ctx->device)) != AUG_OK)
+        return AUG_ECUDA;
     kern<<<grid, FEAT_THREADS, smem, ctx->stream>>>(
         a, b, stride, ctx->gain, table, lengths, c.win, c.hop, c.n_mel, T_max, ctx->melw,
         ctx->melstart, ctx->tw, c.log_floor, c.pad_value, c.compression, out, counts,
@@ -486,7 +488,7 @@ extern "C" int feat_vtlp_logmel_noalloc(const AugConfig *cfg, const float *power
     if (B < 0 || T_max <= 0) return AUG_EINVAL;
     if (cfg->n_fft != 512 && cfg->n_fft != 1024) return AUG_EINVAL;
     if (cfg->n_mel < 1 || cfg->fs <= 0 || !(cfg->f_lo >= 0.f) || !(cfg->f_hi > cfg->f_lo) ||
-        !(cfg->log_floor > 0.f))
+        cfg->f_hi > 0.5f * cfg->fs + 1e-3f || !(cfg->log_floor > 0.f) || !isfinite(cfg->pad_value))
         return AUG_EINVAL;
     if (cfg->compression != AUG_COMPRESS_LOG && cfg->compression != AUG_COMPRESS_POW_1_15)
         return AUG_EINVAL;

@@ -1,21 +1,28 @@
 // Step 1: room impulse responses by the image-source method.
 //
 // One CTA builds one impulse response (one utterance, one source) in shared
-// memory.  Geometry runs in fp64, once per image and spread over the lanes of a
-// warp; the 2*W_h+1 taps of each image are then spread over the lanes in fp32:
-// with tau = n0 + phi, sin(pi (n - tau)) = -(-1)^(n-n0) sin(pi phi), so a tap costs
-// one division and a few FMAs, and the Hann factor comes from the angle-sum
-// identity with per-lane constants.  The lattice points with |kx|+|ky|+|kz| <= order
-// are enumerated compactly (a prefix over kx, then closed forms inside the diamond
-// of (ky, kz)), so every lane of a warp carries a real image.
+// memory.  Every warp works through batches of 32 images in two phases:
+//
+//   A  one image per lane: lattice point, distance and delay in fp64 (the delay
+//      reaches 2.4e4 samples, where one fp32 ulp is 2e-3 samples), split into
+//      an integer n0 and a fraction phi; the five numbers the taps need are
+//      written, compacted over the images that contribute, to a slot of a small
+//      shared-memory ring owned by the warp.
+//   B  one image at a time, its 2 W_h + 1 taps over the lanes: lane l owns taps
+//      l, l + 32, l + 64, so everything that depends only on the tap (its offset,
+//      the cosine and sine of its Hann angle, its sign) sits in registers, and
+//      the image's numbers arrive with two broadcast loads.  With tau = n0 + phi,
+//      sin(pi (n - tau)) = -(-1)^(n - n0) sin(pi phi), and the Hann factor follows
+//      from the angle-sum identity, so a tap costs one reciprocal, three FMAs
+//      and one shared-memory atomic add.
+//
+// The lattice points with |kx|+|ky|+|kz| <= order are enumerated compactly (a
+// prefix over kx, then closed forms inside the diamond of (ky, kz)), so every
+// lane of a warp carries a real image.
 #include "common.cuh"
 
 namespace {
 
-#ifndef RIR_THREADS_N
-#define RIR_THREADS_N 1024
-#endif
-constexpr int RIR_THREADS = RIR_THREADS_N;
 constexpr int AX = 2 * aug::MAX_ORDER + 1;
 
 __device__ __forceinline__ double ipow(double b, int e) {
@@ -24,14 +31,29 @@ __device__ __forceinline__ double ipow(double b, int e) {
     return r;
 }
 
-__global__ void __launch_bounds__(RIR_THREADS)
-rir_image_kernel(const AugUttParams *__restrict__ table, int S_max, int L, int half_w, double fs,
-                 double c, int max_order, int cube, float *__restrict__ rir, int *status) {
+__device__ __forceinline__ float rcp_approx(float x) {
+    float r;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
+}
+
+// Bytes of dynamic shared memory of a CTA of `threads` threads for responses of L taps.
+__host__ __device__ constexpr size_t rir_smem_bytes(int threads, int L) {
+    return sizeof(double) * 3 * AX + sizeof(float) * 3 * AX + sizeof(int) * (AX + 3) +
+           sizeof(float4) * threads + sizeof(float) * threads + sizeof(float) * (size_t)((L + 3) & ~3);
+}
+
+template <int THREADS>
+__global__ void __launch_bounds__(THREADS, 2048 / THREADS)
+rir_image_kernel(const AugUttParams *__restrict__ table, int S_max, int L, int half_w,
+                 double fs_over_c, int max_order, int cube, float *__restrict__ rir, int *status) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    double *dsq = reinterpret_cast<double *>(smem_raw);   // [3][AX]
-    double *gain = dsq + 3 * AX;                          // [3][AX]
-    int *xpre = reinterpret_cast<int *>(gain + 3 * AX);   // [AX + 1] images before slab kx
-    float *h = reinterpret_cast<float *>(xpre + AX + 3);  // [L]
+    float4 *ring4 = reinterpret_cast<float4 *>(smem_raw);          // [THREADS] n0, phi, P0, P1 of an image
+    float *h = reinterpret_cast<float *>(ring4 + THREADS);         // [L rounded up to 4]
+    double *dsq = reinterpret_cast<double *>(h + ((L + 3) & ~3));  // [3][AX] squared coordinate differences
+    float *ring1 = reinterpret_cast<float *>(dsq + 3 * AX);        // [THREADS] P2
+    float *gain = ring1 + THREADS;                                 // [3][AX] wall gains per axis
+    int *xpre = reinterpret_cast<int *>(gain + 3 * AX);            // [AX + 1] images before slab kx
 
     const int utt = blockIdx.y, s = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -43,14 +65,15 @@ rir_image_kernel(const AugUttParams *__restrict__ table, int S_max, int L, int h
     if (n_src < 1 || n_src > S_max) bad = aug::R_NSRC;
     else if (order < 0 || order > max_order) bad = aug::R_ORDER;
     if (bad || s >= n_src) {
-        for (int i = tid; i < L; i += RIR_THREADS) out[i] = 0.f;
+        for (int i = tid; i < L; i += THREADS) out[i] = 0.f;
         if (bad && tid == 0 && s == 0) {
             if (atomicCAS(&status[0], -1, utt) == -1) status[1] = bad;
         }
         return;
     }
 
-    for (int i = tid; i < L; i += RIR_THREADS) h[i] = 0.f;
+    for (int i = tid; i < ((L + 3) >> 2); i += THREADS)
+        reinterpret_cast<float4 *>(h)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     const int side = 2 * order + 1;
     if (tid < 3 * side) {
         const int a = tid / side, k = tid % side - order;
@@ -59,8 +82,8 @@ rir_image_kernel(const AugUttParams *__restrict__ table, int S_max, int L, int h
         const double img = (1 - 2 * p) * (double)row.src_pos[s][a] + 2.0 * m * (double)row.room[a];
         const double diff = img - (double)row.mic[a];
         dsq[a * AX + k + order] = diff * diff;
-        gain[a * AX + k + order] = ipow((double)row.beta[2 * a], abs(m - p)) *
-                                   ipow((double)row.beta[2 * a + 1], abs(m));
+        gain[a * AX + k + order] = (float)(ipow((double)row.beta[2 * a], abs(m - p)) *
+                                           ipow((double)row.beta[2 * a + 1], abs(m)));
     }
     if (tid == 0) {
         int run = 0;
@@ -74,23 +97,29 @@ rir_image_kernel(const AugUttParams *__restrict__ table, int S_max, int L, int h
     __syncthreads();
     const int total = cube ? side * side * side : xpre[side];
 
-    // per-lane tap constants: this lane owns taps j = lane + 32 i - half_w
-    float cj[3], sj[3], sg[3];
+    // Per-lane tap constants: this lane owns taps j = lane + 32 i - half_w, i < 3.  The
+    // sign (-1)^j is the same for all three and is folded into the Hann constants; a
+    // tap beyond 2 half_w gets an offset no window reaches.
+    const float fhw = (float)half_w;
+    const float sgn = ((lane - half_w) & 1) ? -1.f : 1.f;
+    float fj[3], cj[3], sj[3];
 #pragma unroll
     for (int i = 0; i < 3; ++i) {
-        const int j = lane + 32 * i - half_w;
-        cj[i] = cospif((float)j / (float)half_w);
-        sj[i] = sinpif((float)j / (float)half_w);
-        sg[i] = (j & 1) ? -1.f : 1.f;
+        const int jj = lane + 32 * i, j = jj - half_w;
+        fj[i] = jj <= 2 * half_w ? (float)j : 3e9f;
+        cj[i] = sgn * cospif((float)j / fhw);
+        sj[i] = sgn * sinpif((float)j / fhw);
     }
-    const float fhw = (float)half_w;
-    constexpr int NW = RIR_THREADS / 32;
+    constexpr int NW = THREADS / 32;
+    float4 *my4 = ring4 + warp * 32;
+    float *my1 = ring1 + warp * 32;
 
     for (int base = warp * 32; base < total; base += NW * 32) {
+        // ---- phase A: one image per lane
         const int idx = base + lane;
         bool valid = idx < total;
-        int n0 = 0;
-        float phi = 0.f, A = 0.f, As = 0.f, cph = 0.f, sph = 0.f;
+        float4 q = make_float4(0.f, 0.f, 0.f, 0.f);
+        float p2 = 0.f;
         if (valid) {
             int ix, ky, kz;
             if (cube) {
@@ -107,72 +136,95 @@ rir_image_kernel(const AugUttParams *__restrict__ table, int S_max, int L, int h
                 }
                 ix = lo;
                 const int r = order - abs(ix - order);
-                int q = idx - xpre[ix];               // position inside the diamond of radius r
-                // rows ky = -r..0 hold 1, 3, .., 2r+1 points (q < (r+1)^2, row u has u^2 before it);
+                int qq = idx - xpre[ix];              // position inside the diamond of radius r
+                // rows ky = -r..0 hold 1, 3, .., 2r+1 points (qq < (r+1)^2, row u has u^2 before it);
                 // rows ky = 1..r mirror rows r-1..0, counted from the end.
-                const bool upper = q >= (r + 1) * (r + 1);
-                if (upper) q = 2 * r * r + 2 * r - q;
-                int u = (int)sqrtf((float)q);
-                if (u * u > q) --u;
-                if ((u + 1) * (u + 1) <= q) ++u;
+                const bool upper = qq >= (r + 1) * (r + 1);
+                if (upper) qq = 2 * r * r + 2 * r - qq;
+                int u = (int)sqrtf((float)qq);
+                if (u * u > qq) --u;
+                if ((u + 1) * (u + 1) <= qq) ++u;
                 ky = upper ? r - u : u - r;
-                kz = q - u * u - u;
+                kz = qq - u * u - u;
             }
             const int iy = ky + order, iz = kz + order;
-            {
-                const double d = sqrt(dsq[ix] + dsq[AX + iy] + dsq[2 * AX + iz]);
-                const double g = gain[ix] * gain[AX + iy] * gain[2 * AX + iz];
-                const double tau = d * fs / c;
-                const double rt = rint(tau);
-                A = (float)(g / d);
-                valid = (A != 0.f) && (rt - half_w < (double)L);
-                n0 = (int)rt;
-                phi = (float)(tau - rt);
-                As = -A * sinpif(phi) * 0.318309886183790671538f;
-                cph = 0.5f * cospif(phi / fhw);
-                sph = 0.5f * sinpif(phi / fhw);
-            }
+            const double d2 = dsq[ix] + dsq[AX + iy] + dsq[2 * AX + iz];
+            const float g = gain[ix] * gain[AX + iy] * gain[2 * AX + iz];
+            // 1/d from the fp32 reciprocal square root and one Newton step in fp64
+            // (relative error ~1e-14), d = d2/d with one correction
+            double rd = (double)rsqrtf((float)d2);
+            rd = fma(rd, 0.5 * fma(-d2 * rd, rd, 1.0), rd);
+            double d = d2 * rd;
+            d = fma(0.5 * rd, fma(-d, d, d2), d);
+            const double tau = d * fs_over_c;
+            const int n0 = __double2int_rn(tau);
+            float phi = (float)(tau - (double)n0);
+            // a fraction of exactly zero would make the centre tap 0/0: 1e-7 of a sample
+            // away from it the tap is the same to 3e-7 of its size
+            if (fabsf(phi) < 1e-7f) phi = copysignf(1e-7f, phi);
+            const float A = g * (float)rd;
+            valid = d2 > 0.0 && A != 0.f && n0 - half_w < L;
+            const float As = -A * sinpif(phi) * 0.318309886183790671538f;
+            float sps, cps;
+            sincospif(phi / fhw, &sps, &cps);
+            q = make_float4(__int_as_float(n0), phi, 0.5f * As, 0.5f * As * cps);
+            p2 = 0.5f * As * sps;
         }
-        unsigned mask = __ballot_sync(0xffffffffu, valid);
-        while (mask) {
-            const int src = __ffs(mask) - 1;
-            mask &= mask - 1;
-            const int n0b = __shfl_sync(0xffffffffu, n0, src);
-            const float phib = __shfl_sync(0xffffffffu, phi, src);
-            const float Ab = __shfl_sync(0xffffffffu, A, src);
-            const float Asb = __shfl_sync(0xffffffffu, As, src);
-            const float cb = __shfl_sync(0xffffffffu, cph, src);
-            const float sb = __shfl_sync(0xffffffffu, sph, src);
+        const unsigned mask = __ballot_sync(0xffffffffu, valid);
+        if (valid) {
+            const int pos = __popc(mask & ((1u << lane) - 1u));
+            my4[pos] = q;
+            my1[pos] = p2;
+        }
+        __syncwarp();
+        // ---- phase B: the taps of one image over the lanes
+        const int cnt = __popc(mask);
+        for (int k = 0; k < cnt; ++k) {
+            const float4 im = my4[k];
+            const float P2 = my1[k];
+            const int nl = __float_as_int(im.x) + lane - half_w;
+            const float phi = im.y, P0 = sgn * im.z, P1 = im.w;
 #pragma unroll
             for (int i = 0; i < 3; ++i) {
-                const int jj = lane + 32 * i;
-                const int j = jj - half_w;
-                const int n = n0b + j;
-                const float x = (float)j - phib;
-                if (jj <= 2 * half_w && (unsigned)n < (unsigned)L && fabsf(x) <= fhw) {
-                    const float hann = 0.5f + cj[i] * cb + sj[i] * sb;
-                    const float sc = (fabsf(x) < 1e-7f) ? Ab : __fdividef(sg[i] * Asb, x);
-                    atomicAdd(&h[n], sc * hann);
-                }
+                const float x = fj[i] - phi;
+                const int n = nl + 32 * i;
+                // A sinc(x) hann(x) = (1/x) (-A sin(pi phi)/pi) (-1)^j (1/2 + 1/2 cos(pi x / W_h))
+                const float v = rcp_approx(x) * fmaf(sj[i], P2, fmaf(cj[i], P1, P0));
+                if (fabsf(x) <= fhw && (unsigned)n < (unsigned)L) atomicAdd(&h[n], v);
             }
         }
+        __syncwarp();   // the ring slots are rewritten by the next batch
     }
     __syncthreads();
-    for (int i = tid; i < L; i += RIR_THREADS) out[i] = h[i];
+    if ((reinterpret_cast<uintptr_t>(out) & 15) == 0 && (L & 3) == 0) {
+        for (int i = tid; i < (L >> 2); i += THREADS)
+            reinterpret_cast<float4 *>(out)[i] = reinterpret_cast<const float4 *>(h)[i];
+    } else {
+        for (int i = tid; i < L; i += THREADS) out[i] = h[i];
+    }
 }
 
 }  // namespace
 
 int launch_rir(AugCtx *ctx, const AugUttParams *table, int B, float *rir, cudaStream_t st) {
     const AugConfig &c = ctx->cfg;
-    const size_t smem = sizeof(double) * 6 * AX + sizeof(int) * (AX + 3) + sizeof(float) * (size_t)c.rir_taps;
-    // (set on every launch: the attribute belongs to the current device's copy of the kernel)
-    AUG_CUDA_OK(cudaFuncSetAttribute(rir_image_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)smem));
+    // Two CTAs per multiprocessor either way: 1024 threads each while two responses
+    // plus the rings fit in shared memory, 512 for long responses.
+    const size_t per_sm = (size_t)ctx->smem_per_sm;
+    const bool big = 2 * (rir_smem_bytes(1024, c.rir_taps) + 1024) <= per_sm;
+    const size_t smem = rir_smem_bytes(big ? 1024 : 512, c.rir_taps);
+    const double fs_over_c = (double)c.fs / (double)c.sound_speed;
+    const int cube = c.image_lattice == AUG_LATTICE_CUBE ? 1 : 0;
     dim3 grid(c.max_sources, B);
-    rir_image_kernel<<<grid, RIR_THREADS, smem, st>>>(
-        table, c.max_sources, c.rir_taps, c.frac_half_width, (double)c.fs, (double)c.sound_speed,
-        c.max_order, c.image_lattice == AUG_LATTICE_CUBE ? 1 : 0, rir, ctx->status);
+    if (big) {
+        if (smem_opt_in<rir_image_kernel<1024>>(ctx->device) != AUG_OK) return AUG_ECUDA;
+        rir_image_kernel<1024><<<grid, 1024, smem, st>>>(table, c.max_sources, c.rir_taps, c.frac_half_width,
+                                                         fs_over_c, c.max_order, cube, rir, ctx->status);
+    } else {
+        if (smem_opt_in<rir_image_kernel<512>>(ctx->device) != AUG_OK) return AUG_ECUDA;
+        rir_image_kernel<512><<<grid, 512, smem, st>>>(table, c.max_sources, c.rir_taps, c.frac_half_width,
+                                                       fs_over_c, c.max_order, cube, rir, ctx->status);
+    }
     AUG_CUDA_OK(cudaGetLastError());
     ctx->launches++;
     return AUG_OK;

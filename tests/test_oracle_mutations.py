@@ -25,6 +25,7 @@ PIN_CALLS = [
     pins.test_fractional_delay_kernel_delays_a_sinusoid,
     pins.test_delay_kernel_window_shape,
     pins.test_rir_taps_outside_the_buffer_are_dropped,
+    pins.test_two_microphones_on_the_source_axis_differ_by_the_travel_time_of_their_spacing,
     pins.test_conv_hand_case_from_fixture,
     pins.test_conv_delta_is_identity_and_shift,
     lambda: pins.test_conv_matches_library(1000, 37),
@@ -39,6 +40,7 @@ PIN_CALLS = [
     pins.test_stft_window_is_periodic_hann,
     lambda: pins.test_warp_is_the_phase_of_a_first_order_allpass(0.8),
     lambda: pins.test_warp_is_the_phase_of_a_first_order_allpass(1.2),
+    pins.test_mel_scale_points_from_fixture,
     lambda: pins.test_mel_alpha_one_is_the_unwarped_filterbank(512, 40),
     lambda: pins.test_mel_partition_of_unity(0.9),
     lambda: pins.test_pure_tone_peaks_in_the_band_of_its_warped_frequency(0.8),
@@ -144,3 +146,18 @@ def test_python_mutation_is_caught(name, monkeypatch):
     attr, fn = PY_MUTATIONS[name]
     monkeypatch.setattr(oracle, attr, fn)
     assert failures() >= 1, f"no pin noticed: {name}"
+
+
+def test_mel_scale_mutations_are_caught_by_the_numeric_pin_alone(monkeypatch):
+    # the other mel tests call oracle.hz_to_mel on both sides or retype its formula;
+    # the fixture of hand-worked points must notice a wrong break frequency, a wrong
+    # constant and a natural logarithm by itself
+    pins.test_mel_scale_points_from_fixture()
+    wrong = [_mut_mel,
+             lambda f: 1127.0 * np.log10(1.0 + np.asarray(f, dtype=np.float64) / 700.0),
+             lambda f: 2595.0 * np.log(1.0 + np.asarray(f, dtype=np.float64) / 700.0),
+             lambda f: 2595.0 * np.log10(np.asarray(f, dtype=np.float64) / 700.0 + 1e-300)]
+    for fn in wrong:
+        monkeypatch.setattr(oracle, "hz_to_mel", fn)
+        with pytest.raises(AssertionError):
+            pins.test_mel_scale_points_from_fixture()

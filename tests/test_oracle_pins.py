@@ -159,6 +159,31 @@ def test_delay_kernel_window_shape():
     assert abs(h[n0 + 21]) == pytest.approx(0.5 / (20.5 * np.pi), rel=1e-9)
 
 
+def test_two_microphones_on_the_source_axis_differ_by_the_travel_time_of_their_spacing():
+    # The far-field set-up of the paper's Section 4 (Fig. 4): source 5 m from a pair of
+    # microphones 6.8 cm apart.  Without reflections and with the source on the array
+    # axis, the second channel is the first one delayed by 0.068 fs / c = 3.172 samples
+    # and weaker by the ratio of the distances.  The delay is read off the phase slope
+    # of the response at low frequency, the level off its value near DC.
+    room = [12.0, 6.0, 3.0]
+    src = [1.0, 3.0, 1.5]
+    mics = ([6.0, 3.0, 1.5], [6.068, 3.0, 1.5])
+    L = 1024
+    k = np.arange(L)
+    w1, w2 = 2 * np.pi * 0.040, 2 * np.pi * 0.041          # (w2 - w1) tau = 1.5 < pi: no phase wrap
+    tau, level = [], []
+    for mic in mics:
+        h = oracle.rir_image_method(room, [0.0] * 6, mic, src, 3, L)
+        H1, H2 = np.sum(h * np.exp(-1j * w1 * k)), np.sum(h * np.exp(-1j * w2 * k))
+        tau.append(-np.angle(H2 / H1) / (w2 - w1))
+        level.append(abs(np.sum(h * np.exp(-1j * 2 * np.pi * 0.01 * k))))
+    assert tau[0] == pytest.approx(5.0 * FS / C, abs=1e-3)
+    assert tau[1] - tau[0] == pytest.approx(0.068 * FS / C, abs=1e-3)        # 3.172 samples
+    assert 3.17 < tau[1] - tau[0] < 3.175
+    assert level[0] / level[1] == pytest.approx(5.068 / 5.0, rel=1e-4)
+    assert level[0] == pytest.approx(1 / 5.0, rel=1e-3)
+
+
 def test_rir_taps_outside_the_buffer_are_dropped():
     room, mic, src = [5.0, 4.0, 3.0], [1.0, 1.2, 1.1], [3.3, 2.9, 1.7]
     beta = [0.8] * 6
@@ -295,6 +320,16 @@ def test_warp_is_the_phase_of_a_first_order_allpass(alpha):
         assert np.all(got[1:-1] > w[1:-1])      # alpha < 1 moves content upward
     if alpha == 1.0:
         np.testing.assert_array_equal(got, w)
+
+
+def test_mel_scale_points_from_fixture():
+    # numbers, not the formula again: 700 Hz is 2595 log10(2) mel, 1000 Hz is the
+    # scale's anchor (1000 mel to 0.0015 %), 6300 Hz is 2595 mel
+    pts = np.loadtxt(os.path.join(GOLD, "mel_scale_points.txt"))
+    assert pts.shape == (4, 2)
+    np.testing.assert_allclose(oracle.hz_to_mel(pts[:, 0]), pts[:, 1], atol=1e-3)
+    # 1000 mel at 1000 Hz is what the constant 2595 was chosen for
+    assert abs(float(oracle.hz_to_mel(1000.0)) - 1000.0) < 0.02
 
 
 def _plain_mel(n_fft, n_mel, fs):
