@@ -331,6 +331,260 @@ frames_kernel(const float *__restrict__ in_a, const float *__restrict__ in_b, in
     }
 }
 
+// ---------------------------------------------------------------- fused path, one warp per frame pair
+// 512-point transforms of the fused path.  A warp takes a frame pair from its
+// samples to its two power spectra: lane t holds 16 of the 512 complex points
+// (frame 2p in the real, frame 2p+1 in the imaginary part) as two radix-8
+// butterflies per pass, exchanges them through a buffer of its own (warp barriers
+// only), and in the last pass takes butterflies t and 64-t, whose outputs are the
+// bins k and 512-k: the two spectra are separated and squared in registers and
+// only the powers go to shared memory.  A CTA of eight warps does a tile of 16
+// frames at a time; the filterbank then runs with the frames of the tile over the
+// lanes (every edge interval walked once, all lanes on the same bins), while the
+// samples of the next tile are already on their way from global memory.
+namespace wp {
+
+constexpr int K = 512;
+constexpr int NBP = K / 2 + 1;
+constexpr int XB = padded_points(K);          // float2 slots of a warp's exchange buffer
+constexpr int WARPS = FEAT_THREADS / 32;
+constexpr int FT = 2 * WARPS;                  // frames per tile: one pair per warp
+constexpr int SV = 3;                          // 128-bit staging loads per thread, array and tile
+
+template <int NS>
+__device__ __forceinline__ void scatter8(const float2 *v, float2 *s, int j) {
+    constexpr int PS = out_shift(NS);
+    const int k = j & (NS - 1);
+    const int base = padi<PS>((j - k) * 8 + k);
+#pragma unroll
+    for (int r = 0; r < 8; ++r) s[base + padi<PS>(r * NS)] = v[r];
+}
+
+// |A|^2 and |B|^2 at bin k from Z[k] = z and Z[K-k] = q, where Z is the transform of a + i b.
+__device__ __forceinline__ void power_pair(float2 z, float2 q, float &pa, float &pb) {
+    const float ar = z.x + q.x, ai = z.y - q.y;
+    const float br = z.y + q.y, bi = z.x - q.x;
+    pa = 0.25f * fmaf(ar, ar, ai * ai);
+    pb = 0.25f * fmaf(br, br, bi * bi);
+}
+
+__host__ __device__ constexpr int chunk_floats(int win, int hop) { return ((FT - 1) * hop + win + 3) & ~3; }
+__host__ __device__ constexpr size_t smem_bytes(int win, int hop, int M) {
+    return sizeof(float2) * WARPS * XB + sizeof(float) * FT * NBP + sizeof(float) * chunk_floats(win, hop) +
+           sizeof(float) * K + sizeof(float2) * (NBP + 1) + sizeof(int) * (M + 2);
+}
+
+template <int TILES>
+__global__ void __launch_bounds__(FEAT_THREADS, FEAT_MINB)
+frames_warp_kernel(const float *__restrict__ in_a, const float *__restrict__ in_b, int64_t in_stride,
+                   const float *__restrict__ gain, const int *__restrict__ lengths, int win, int hop,
+                   int M, int T_max, const aug::MelBin *__restrict__ melw,
+                   const int *__restrict__ melstart, const float2 *__restrict__ tw, float floor_v,
+                   float pad_v, int comp, float *__restrict__ out, int *__restrict__ counts, int n_cap) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int chunk_cap = chunk_floats(win, hop);
+    float2 *xb_all = reinterpret_cast<float2 *>(smem_raw);                   // [WARPS][XB]; later the interval sums
+    float *ptile = reinterpret_cast<float *>(xb_all + WARPS * XB);           // [FT][NBP]
+    float *chunk = ptile + FT * NBP;                                         // [chunk_cap]
+    float *win_s = chunk + chunk_cap;                                        // [K] Hann, zero beyond win
+    float2 *mw = reinterpret_cast<float2 *>(win_s + K);                      // [NBP + 1] (up, down)
+    int *mst = reinterpret_cast<int *>(mw + NBP + 1);                        // [M + 2]
+
+    const int utt = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int run0 = blockIdx.x * (FT * TILES);
+    const int N = min(max(lengths[utt], 0), n_cap);
+    const int T = min(frame_count(N, win, hop), T_max);
+    if (blockIdx.x == 0 && tid == 0) counts[utt] = T;
+    const int rows = min(FT * TILES, T_max - run0);
+    if (rows <= 0) return;
+    const int nfr = max(0, min(FT * TILES, T - run0));
+    float *orun = out + ((int64_t)utt * T_max + run0) * M;
+    for (int i = nfr * M + tid; i < rows * M; i += FEAT_THREADS) orun[i] = pad_v;
+    if (nfr == 0) return;
+
+    const float g = gain[utt];
+    const float *ra = in_a + (int64_t)utt * in_stride;
+    const float *rb = in_b + (int64_t)utt * in_stride;
+    // 128-bit staging needs 16-byte aligned tile starts and at most SV loads per thread
+    const bool vec = (hop & 3) == 0 && (in_stride & 3) == 0 && chunk_cap <= SV * FEAT_THREADS * 4;
+    for (int n = tid; n < K; n += FEAT_THREADS)
+        win_s[n] = n < win ? 0.5f - 0.5f * cospif(2.f * (float)n / (float)win) : 0.f;
+    for (int k = tid; k < NBP; k += FEAT_THREADS) {
+        const aug::MelBin w = melw[(int64_t)utt * NBP + k];
+        mw[k] = make_float2(w.up, w.down);
+    }
+    for (int m = tid; m < M + 2; m += FEAT_THREADS) mst[m] = melstart[(int64_t)utt * (M + 2) + m];
+
+    // Lane constants: twiddles of the last pass for this lane's two butterflies
+    // (j0 = lane and its mirror j1 = 64 - lane; lane 0 takes the self-mirrored 0 and 32)
+    // and the first twiddle of the middle pass.
+    const int j0 = lane, j1 = lane ? 64 - lane : 32;
+    float2 w3a[8], w3b[8];
+    twiddle_powers<8>(w3a, __ldg(&tw[tw_index(K, j0)]));
+    twiddle_powers<8>(w3b, __ldg(&tw[tw_index(K, j1)]));
+    const float2 w2_1 = __ldg(&tw[tw_index(64, lane & 7)]);
+    float2 *xb = xb_all + warp * XB;
+    float *up_s = reinterpret_cast<float *>(xb_all);         // [FT][M + 1] rising sums (transforms are done)
+    float *dn_s = up_s + FT * (M + 1);                       // [FT][M + 1] falling sums
+    const int n_tiles = min(TILES, (nfr + FT - 1) / FT);
+
+    // samples of a tile: loaded into registers (all loads in flight together), mixed and
+    // stored to `chunk` one phase later
+    float4 xa[SV], xv[SV];
+    auto stage_load = [&](int tile) {
+        const int s0 = (run0 + tile * FT) * hop;
+        const int ns = (min(FT, T - (run0 + tile * FT)) - 1) * hop + win;
+#pragma unroll
+        for (int u = 0; u < SV; ++u) {
+            const int i = (tid + u * FEAT_THREADS) * 4;
+            xa[u] = xv[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (i < ns) {      // rows are allocated up to a multiple of 4 floats: whole groups can be read
+                xa[u] = __ldg(reinterpret_cast<const float4 *>(ra + s0 + i));
+                if (g != 0.f) xv[u] = __ldg(reinterpret_cast<const float4 *>(rb + s0 + i));
+            }
+        }
+    };
+    auto stage_store = [&]() {
+#pragma unroll
+        for (int u = 0; u < SV; ++u) {
+            const int i = (tid + u * FEAT_THREADS) * 4;
+            if (i < chunk_cap)
+                *reinterpret_cast<float4 *>(chunk + i) =
+                    make_float4(fmaf(g, xv[u].x, xa[u].x), fmaf(g, xv[u].y, xa[u].y),
+                                fmaf(g, xv[u].z, xa[u].z), fmaf(g, xv[u].w, xa[u].w));
+        }
+    };
+    auto stage_scalar = [&](int tile) {
+        const int s0 = (run0 + tile * FT) * hop;
+        const int ns = (min(FT, T - (run0 + tile * FT)) - 1) * hop + win;
+        for (int i = tid; i < ns; i += FEAT_THREADS)
+            chunk[i] = g != 0.f ? fmaf(g, rb[s0 + i], ra[s0 + i]) : ra[s0 + i];
+    };
+    if (vec) stage_load(0);
+
+    for (int tile = 0; tile < n_tiles; ++tile) {
+        const int t0 = run0 + tile * FT;
+        const int nf = min(FT, T - t0);
+        if (vec) stage_store(); else stage_scalar(tile);
+        __syncthreads();                      // chunk (and, first time, the tables) in place; sums of the last tile read
+
+        const int f0 = 2 * warp;
+        if (f0 < nf) {
+            const bool have1 = f0 + 1 < nf;
+            const float *c0 = chunk + f0 * hop;
+            float2 v[2][8];
+            // butterfly b of the first pass is j = lane + 32 b: points j + 64 r
+#pragma unroll
+            for (int b = 0; b < 2; ++b) {
+#pragma unroll
+                for (int r = 0; r < 8; ++r) {
+                    const int n = lane + 32 * (2 * r + b);
+                    float a = 0.f, bb = 0.f;
+                    if (n < win) {
+                        const float wn = win_s[n];
+                        a = wn * c0[n];
+                        if (have1) bb = wn * c0[hop + n];
+                    }
+                    v[b][r] = make_float2(a, bb);
+                }
+            }
+            Dft<8>::run(v[0]);
+            Dft<8>::run(v[1]);
+            scatter8<1>(v[0], xb, lane);
+            scatter8<1>(v[1], xb, lane + 32);
+            __syncwarp();
+            gather<K, 16, 8, 1>(v, xb, lane);
+            __syncwarp();
+            {
+                float2 w2[8];
+                twiddle_powers<8>(w2, w2_1);
+#pragma unroll
+                for (int r = 1; r < 8; ++r) {
+                    v[0][r] = cmul(v[0][r], w2[r]);
+                    v[1][r] = cmul(v[1][r], w2[r]);
+                }
+            }
+            Dft<8>::run(v[0]);
+            Dft<8>::run(v[1]);
+            scatter8<8>(v[0], xb, lane);
+            scatter8<8>(v[1], xb, lane + 32);
+            __syncwarp();
+            {
+                constexpr int PS = out_shift(8);
+                const int b0 = padi<PS>(j0), b1 = padi<PS>(j1);
+#pragma unroll
+                for (int r = 0; r < 8; ++r) {
+                    v[0][r] = xb[b0 + padi<PS>(r * 64)];
+                    v[1][r] = xb[b1 + padi<PS>(r * 64)];
+                }
+            }
+#pragma unroll
+            for (int r = 1; r < 8; ++r) {
+                v[0][r] = cmul(v[0][r], w3a[r]);
+                v[1][r] = cmul(v[1][r], w3b[r]);
+            }
+            Dft<8>::run(v[0]);     // bins j0 + 64 r
+            Dft<8>::run(v[1]);     // bins j1 + 64 r
+            // Bin k pairs with bin 512 - k: for j0 + 64 r that is output 7 - r of the other
+            // butterfly (lane 0: butterfly 0 pairs with itself, 64 r with 64 (8 - r), and so
+            // does butterfly 32).  Only bins up to 256 are kept.
+            float *p0 = ptile + f0 * NBP, *p1 = p0 + NBP;
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                const float2 qa = lane ? v[1][7 - r] : v[0][(8 - r) & 7];
+                const float2 qb = lane ? v[0][7 - r] : v[1][7 - r];
+                float pa, pb;
+                power_pair(v[0][r], qa, pa, pb);
+                p0[j0 + 64 * r] = pa;
+                if (have1) p1[j0 + 64 * r] = pb;
+                power_pair(v[1][r], qb, pa, pb);
+                p0[j1 + 64 * r] = pa;
+                if (have1) p1[j1 + 64 * r] = pb;
+            }
+            if (lane == 0) {
+                float pa, pb;
+                power_pair(v[0][4], v[0][4], pa, pb);
+                p0[K / 2] = pa;
+                if (have1) p1[K / 2] = pb;
+            }
+        }
+        __syncthreads();                      // power spectra of the tile in place; chunk and the buffers are free
+        if (vec && tile + 1 < n_tiles) stage_load(tile + 1);
+
+        // Filterbank with the frames of the tile over the lanes, two edge intervals per
+        // warp step: the bins of interval j give its rising sum (band j) and its falling
+        // sum (band j-1).
+        {
+            const int f = lane & (FT - 1), sub = lane / FT;
+            constexpr int BPW = 32 / FT;
+            for (int jb = warp * BPW; jb <= M; jb += WARPS * BPW) {
+                const int j = jb + sub;
+                if (j <= M && f < nf) {
+                    const float *p = ptile + f * NBP;
+                    float u = 0.f, d = 0.f;
+                    const int k1 = mst[j + 1];
+                    for (int k = mst[j]; k < k1; ++k) {
+                        const float2 w = mw[k];
+                        const float pk = p[k];
+                        u = fmaf(w.x, pk, u);
+                        d = fmaf(w.y, pk, d);
+                    }
+                    up_s[f * (M + 1) + j] = u;
+                    dn_s[f * (M + 1) + j] = d;
+                }
+            }
+        }
+        __syncthreads();                      // interval sums in place
+        float *orow = orun + (int64_t)tile * FT * M;
+        for (int i = tid; i < nf * M; i += FEAT_THREADS) {
+            const int ff = i / M, m = i - ff * M;
+            orow[i] = compress(up_s[ff * (M + 1) + m] + dn_s[ff * (M + 1) + m + 1], floor_v, comp);
+        }
+    }
+}
+
+}  // namespace wp
+
 // ---------------------------------------------------------------- step 4 alone
 __global__ void __launch_bounds__(256)
 logmel_kernel(const float *__restrict__ power, const int *__restrict__ counts, int NBP, int M,
@@ -408,9 +662,38 @@ int launch_stft_power(AugCtx *ctx, const float *wave, int64_t stride, const int 
     return launch_frames<1024, 0>(ctx, wave, nullptr, stride, lengths, nullptr, B, power, T_max, counts);
 }
 
+#ifndef FEAT_WP_TILES
+#define FEAT_WP_TILES 8     // consecutive 16-frame tiles one CTA of the warp-per-pair kernel works through
+#endif
+
+// Fused features with the 512-point transform: the warp-per-frame-pair kernel.
+static int launch_frames_warp(AugCtx *ctx, const int *lengths, int B, float *feats, int T_max, int *counts) {
+    const AugConfig &c = ctx->cfg;
+    const size_t smem = wp::smem_bytes(c.win, c.hop, c.n_mel);
+    if (smem > 227 * 1024) return AUG_ECAP;
+    const int n_tiles = (T_max + wp::FT - 1) / wp::FT;
+    const bool runs = (int64_t)n_tiles * B >= 2 * (int64_t)ctx->sm_count * FEAT_WP_TILES;
+    const int RUN = wp::FT * (runs ? FEAT_WP_TILES : 1);
+    dim3 grid((T_max + RUN - 1) / RUN, B);
+    auto kern = runs ? wp::frames_warp_kernel<FEAT_WP_TILES> : wp::frames_warp_kernel<1>;
+    if ((runs ? smem_opt_in<wp::frames_warp_kernel<FEAT_WP_TILES>>(ctx->device)
+              : smem_opt_in<wp::frames_warp_kernel<1>>(ctx->device)) != AUG_OK)
+        return AUG_ECUDA;
+    kern<<<grid, FEAT_THREADS, smem, ctx->stream>>>(
+        ctx->ys, ctx->vv, ctx->ws_stride, ctx->gain, lengths, c.win, c.hop, c.n_mel, T_max, ctx->melw,
+        ctx->melstart, ctx->tw, c.log_floor, c.pad_value, c.compression, feats, counts,
+        (int)(ctx->ws_stride < 0x7fffffff ? ctx->ws_stride : 0x7fffffff));
+    AUG_CUDA_OK(cudaGetLastError());
+    ctx->launches++;
+    return AUG_OK;
+}
+
 int launch_fused_features(AugCtx *ctx, const int *lengths, const AugUttParams *table, int B,
                           float *feats, int T_max, int *counts) {
     if (T_max <= 0) return AUG_OK;
+#ifndef FEAT_OLD_512
+    if (ctx->cfg.n_fft == 512) return launch_frames_warp(ctx, lengths, B, feats, T_max, counts);
+#endif
     if (ctx->cfg.n_fft == 512)
         return launch_frames<512, 1>(ctx, ctx->ys, ctx->vv, ctx->ws_stride, lengths, table, B, feats,
                                      T_max, counts);

@@ -14,7 +14,17 @@
 //      the image's numbers arrive with two broadcast loads.  With tau = n0 + phi,
 //      sin(pi (n - tau)) = -(-1)^(n - n0) sin(pi phi), and the Hann factor follows
 //      from the angle-sum identity, so a tap costs one reciprocal, three FMAs
-//      and one shared-memory atomic add.
+//      and one shared-memory reduction.
+//
+// The response is accumulated in 32-bit fixed point: a shared-memory fp32 atomic
+// add is a compare-and-swap loop on this hardware, an integer one is a single
+// instruction.  The scale is a power of two chosen per response from the direct
+// path, the largest single contribution (A0 = 1/d0): full scale is 64 A0, one
+// step 3e-8 A0 (coarser steps show in narrow mel bands that fall into a notch of
+// the room's transfer function).  Integer sums are exact, so only the final value
+// of a sample has to fit: with fully reflecting walls and order 32 the largest
+// sample is 2-3 A0 in rooms of a few metres and 14 A0 in a 30 cm box; a sample
+// beyond 64 A0 (rooms of a few centimetres) would wrap.
 //
 // The lattice points with |kx|+|ky|+|kz| <= order are enumerated compactly (a
 // prefix over kx, then closed forms inside the diamond of (ky, kz)), so every
@@ -37,19 +47,40 @@ __device__ __forceinline__ float rcp_approx(float x) {
     return r;
 }
 
+// Add v, rounded to the nearest integer, to the int at shared address a + OFF if
+// |x| <= lim, as one predicated instruction (no branch around it).
+template <int OFF>
+__device__ __forceinline__ void red_shared_within(unsigned a, float v, float x, float lim) {
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        ".reg .f32 ax;\n\t"
+        "abs.f32 ax, %2;\n\t"
+        "setp.le.f32 p, ax, %3;\n\t"
+        ".reg .s32 iv;\n\t"
+        "cvt.rni.s32.f32 iv, %1;\n\t"
+        "@p red.shared.add.s32 [%0+%4], iv;\n\t"
+        "}"
+        :
+        : "r"(a), "f"(v), "f"(x), "f"(lim), "n"(OFF)
+        : "memory");
+}
+
 // Bytes of dynamic shared memory of a CTA of `threads` threads for responses of L taps.
 __host__ __device__ constexpr size_t rir_smem_bytes(int threads, int L) {
     return sizeof(double) * 3 * AX + sizeof(float) * 3 * AX + sizeof(int) * (AX + 3) +
            sizeof(float4) * threads + sizeof(float) * threads + sizeof(float) * (size_t)((L + 3) & ~3);
 }
 
-template <int THREADS>
-__global__ void __launch_bounds__(THREADS, 2048 / THREADS)
+constexpr int THREADS = 512;      // 16 warps; two or three CTAs per multiprocessor
+constexpr float HEADROOM_LOG2 = 6.f;   // full scale = 2^6 times the direct-path amplitude
+
+__global__ void __launch_bounds__(THREADS, 3)
 rir_image_kernel(const AugUttParams *__restrict__ table, int S_max, int L, int half_w,
                  double fs_over_c, int max_order, int cube, float *__restrict__ rir, int *status) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float4 *ring4 = reinterpret_cast<float4 *>(smem_raw);          // [THREADS] n0, phi, P0, P1 of an image
-    float *h = reinterpret_cast<float *>(ring4 + THREADS);         // [L rounded up to 4]
+    int *h = reinterpret_cast<int *>(ring4 + THREADS);             // [L rounded up to 4] fixed-point response
     double *dsq = reinterpret_cast<double *>(h + ((L + 3) & ~3));  // [3][AX] squared coordinate differences
     float *ring1 = reinterpret_cast<float *>(dsq + 3 * AX);        // [THREADS] P2
     float *gain = ring1 + THREADS;                                 // [3][AX] wall gains per axis
@@ -72,8 +103,7 @@ rir_image_kernel(const AugUttParams *__restrict__ table, int S_max, int L, int h
         return;
     }
 
-    for (int i = tid; i < ((L + 3) >> 2); i += THREADS)
-        reinterpret_cast<float4 *>(h)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int i = tid; i < ((L + 3) >> 2); i += THREADS) reinterpret_cast<int4 *>(h)[i] = make_int4(0, 0, 0, 0);
     const int side = 2 * order + 1;
     if (tid < 3 * side) {
         const int a = tid / side, k = tid % side - order;
@@ -96,6 +126,10 @@ rir_image_kernel(const AugUttParams *__restrict__ table, int S_max, int L, int h
     }
     __syncthreads();
     const int total = cube ? side * side * side : xpre[side];
+    // fixed-point scale: a power of two with 2^31 / scale >= 2^HEADROOM_LOG2 / d0
+    const float d0sq = (float)(dsq[order] + dsq[AX + order] + dsq[2 * AX + order]);
+    const float e2 = d0sq > 0.f ? floorf(31.f - HEADROOM_LOG2 + 0.5f * log2f(d0sq)) : 0.f;
+    const float scale = exp2f(fminf(fmaxf(e2, -60.f), 60.f)), inv_scale = exp2f(-fminf(fmaxf(e2, -60.f), 60.f));
 
     // Per-lane tap constants: this lane owns taps j = lane + 32 i - half_w, i < 3.  The
     // sign (-1)^j is the same for all three and is folded into the Hann constants; a
@@ -111,6 +145,8 @@ rir_image_kernel(const AugUttParams *__restrict__ table, int S_max, int L, int h
         sj[i] = sgn * sinpif((float)j / fhw);
     }
     constexpr int NW = THREADS / 32;
+    const unsigned h_addr = (unsigned)__cvta_generic_to_shared(h);
+    const unsigned inside = (unsigned)max(L - 2 * half_w, 0);   // first-tap samples whose whole window fits
     float4 *my4 = ring4 + warp * 32;
     float *my1 = ring1 + warp * 32;
 
@@ -164,7 +200,7 @@ rir_image_kernel(const AugUttParams *__restrict__ table, int S_max, int L, int h
             if (fabsf(phi) < 1e-7f) phi = copysignf(1e-7f, phi);
             const float A = g * (float)rd;
             valid = d2 > 0.0 && A != 0.f && n0 - half_w < L;
-            const float As = -A * sinpif(phi) * 0.318309886183790671538f;
+            const float As = -A * scale * sinpif(phi) * 0.318309886183790671538f;
             float sps, cps;
             sincospif(phi / fhw, &sps, &cps);
             q = make_float4(__int_as_float(n0), phi, 0.5f * As, 0.5f * As * cps);
@@ -182,25 +218,38 @@ rir_image_kernel(const AugUttParams *__restrict__ table, int S_max, int L, int h
         for (int k = 0; k < cnt; ++k) {
             const float4 im = my4[k];
             const float P2 = my1[k];
-            const int nl = __float_as_int(im.x) + lane - half_w;
+            const int n_first = __float_as_int(im.x) - half_w;      // sample of tap -half_w
             const float phi = im.y, P0 = sgn * im.z, P1 = im.w;
+            // A sinc(x) hann(x) = (1/x) (-A sin(pi phi)/pi) (-1)^j (1/2 + 1/2 cos(pi x / W_h)), x = j - phi
+            if ((unsigned)n_first < inside) {
+                // every tap of the window falls inside the response: no index checks, the
+                // three adds go to fixed offsets from one address
+                const unsigned a = h_addr + 4u * (unsigned)(n_first + lane);
+                const float x0 = fj[0] - phi, x1 = fj[1] - phi, x2 = fj[2] - phi;
+                red_shared_within<0>(a, rcp_approx(x0) * fmaf(sj[0], P2, fmaf(cj[0], P1, P0)), x0, fhw);
+                red_shared_within<128>(a, rcp_approx(x1) * fmaf(sj[1], P2, fmaf(cj[1], P1, P0)), x1, fhw);
+                red_shared_within<256>(a, rcp_approx(x2) * fmaf(sj[2], P2, fmaf(cj[2], P1, P0)), x2, fhw);
+            } else {
 #pragma unroll
-            for (int i = 0; i < 3; ++i) {
-                const float x = fj[i] - phi;
-                const int n = nl + 32 * i;
-                // A sinc(x) hann(x) = (1/x) (-A sin(pi phi)/pi) (-1)^j (1/2 + 1/2 cos(pi x / W_h))
-                const float v = rcp_approx(x) * fmaf(sj[i], P2, fmaf(cj[i], P1, P0));
-                if (fabsf(x) <= fhw && (unsigned)n < (unsigned)L) atomicAdd(&h[n], v);
+                for (int i = 0; i < 3; ++i) {
+                    const float x = fj[i] - phi;
+                    const int n = n_first + lane + 32 * i;
+                    const float v = rcp_approx(x) * fmaf(sj[i], P2, fmaf(cj[i], P1, P0));
+                    if (fabsf(x) <= fhw && (unsigned)n < (unsigned)L) atomicAdd(&h[n], __float2int_rn(v));
+                }
             }
         }
         __syncwarp();   // the ring slots are rewritten by the next batch
     }
     __syncthreads();
     if ((reinterpret_cast<uintptr_t>(out) & 15) == 0 && (L & 3) == 0) {
-        for (int i = tid; i < (L >> 2); i += THREADS)
-            reinterpret_cast<float4 *>(out)[i] = reinterpret_cast<const float4 *>(h)[i];
+        for (int i = tid; i < (L >> 2); i += THREADS) {
+            const int4 q = reinterpret_cast<const int4 *>(h)[i];
+            reinterpret_cast<float4 *>(out)[i] = make_float4((float)q.x * inv_scale, (float)q.y * inv_scale,
+                                                             (float)q.z * inv_scale, (float)q.w * inv_scale);
+        }
     } else {
-        for (int i = tid; i < L; i += THREADS) out[i] = h[i];
+        for (int i = tid; i < L; i += THREADS) out[i] = (float)h[i] * inv_scale;
     }
 }
 
@@ -208,23 +257,13 @@ rir_image_kernel(const AugUttParams *__restrict__ table, int S_max, int L, int h
 
 int launch_rir(AugCtx *ctx, const AugUttParams *table, int B, float *rir, cudaStream_t st) {
     const AugConfig &c = ctx->cfg;
-    // Two CTAs per multiprocessor either way: 1024 threads each while two responses
-    // plus the rings fit in shared memory, 512 for long responses.
-    const size_t per_sm = (size_t)ctx->smem_per_sm;
-    const bool big = 2 * (rir_smem_bytes(1024, c.rir_taps) + 1024) <= per_sm;
-    const size_t smem = rir_smem_bytes(big ? 1024 : 512, c.rir_taps);
+    const size_t smem = rir_smem_bytes(THREADS, c.rir_taps);
     const double fs_over_c = (double)c.fs / (double)c.sound_speed;
     const int cube = c.image_lattice == AUG_LATTICE_CUBE ? 1 : 0;
     dim3 grid(c.max_sources, B);
-    if (big) {
-        if (smem_opt_in<rir_image_kernel<1024>>(ctx->device) != AUG_OK) return AUG_ECUDA;
-        rir_image_kernel<1024><<<grid, 1024, smem, st>>>(table, c.max_sources, c.rir_taps, c.frac_half_width,
-                                                         fs_over_c, c.max_order, cube, rir, ctx->status);
-    } else {
-        if (smem_opt_in<rir_image_kernel<512>>(ctx->device) != AUG_OK) return AUG_ECUDA;
-        rir_image_kernel<512><<<grid, 512, smem, st>>>(table, c.max_sources, c.rir_taps, c.frac_half_width,
-                                                       fs_over_c, c.max_order, cube, rir, ctx->status);
-    }
+    if (smem_opt_in<rir_image_kernel>(ctx->device) != AUG_OK) return AUG_ECUDA;
+    rir_image_kernel<<<grid, THREADS, smem, st>>>(table, c.max_sources, c.rir_taps, c.frac_half_width,
+                                                  fs_over_c, c.max_order, cube, rir, ctx->status);
     AUG_CUDA_OK(cudaGetLastError());
     ctx->launches++;
     return AUG_OK;

@@ -110,6 +110,31 @@ def test_two_microphone_array_as_paired_rows():
         assert np.max(np.abs(h[2 * u, 0] - h[2 * u + 1, 0])) > 1e-3 * np.max(np.abs(h[2 * u, 0]))
 
 
+@pytest.mark.parametrize("dist", [0.05, 1.0, 60.0])
+def test_rir_accumulation_scale_follows_the_direct_path(dist):
+    """The response is accumulated in fixed point scaled to the direct sound: a source
+    5 cm from the microphone (amplitude 20) and one 60 m away (amplitude 0.017) must
+    both come out within the same relative tolerance."""
+    w = small(2, batch=2, dur_scale=0.05, order=6)
+    for b in range(w.B):
+        row = w.table[b]
+        row["room"] = (80.0, 9.0, 4.0)
+        row["beta"] = (0.9, 0.8, 0.85, 0.7, 0.6, 0.75)
+        row["mic"] = (5.0, 4.0, 1.5)
+        row["n_src"] = 2
+        row["src_pos"][0] = (5.0 + dist, 4.0, 1.5)
+        row["src_pos"][1] = (5.0 + dist * 0.6, 4.0 + dist * 0.05, 1.5 + min(dist, 2.0) * 0.4)
+    dev = Device(w)
+    h = dev.rir().cpu().numpy()
+    for b in range(w.B):
+        row = w.table[b]
+        for s in range(2):
+            ref = oracle.rir_image_method(row["room"], row["beta"], row["mic"], row["src_pos"][s],
+                                          int(row["order"]), dev.L)
+            assert np.max(np.abs(ref)) > 0
+            assert np.max(np.abs(h[b, s] - ref)) <= RIR_REL_TOL * np.max(np.abs(ref)), (dist, b, s)
+
+
 def test_rir_closed_form_single_image():
     w = small(1, batch=1, dur_scale=0.05)
     row = w.table[0]
