@@ -407,6 +407,8 @@ frames_warp_kernel(const float *__restrict__ in_a, const float *__restrict__ in_
     const float *rb = in_b + (int64_t)utt * in_stride;
     // 128-bit staging needs 16-byte aligned tile starts and at most SV loads per thread
     const bool vec = (hop & 3) == 0 && (in_stride & 3) == 0 && chunk_cap <= SV * FEAT_THREADS * 4;
+    // 64-bit loads of sample pairs: frames start on even samples and the window ends on one
+    const bool pairs = ((hop | win) & 1) == 0 && win >= 2;
     for (int n = tid; n < K; n += FEAT_THREADS)
         win_s[n] = n < win ? 0.5f - 0.5f * cospif(2.f * (float)n / (float)win) : 0.f;
     for (int k = tid; k < NBP; k += FEAT_THREADS) {
@@ -427,6 +429,8 @@ frames_warp_kernel(const float *__restrict__ in_a, const float *__restrict__ in_
     float *up_s = reinterpret_cast<float *>(xb_all);         // [FT][M + 1] rising sums (transforms are done)
     float *dn_s = up_s + FT * (M + 1);                       // [FT][M + 1] falling sums
     const int n_tiles = min(TILES, (nfr + FT - 1) / FT);
+    const int out_f0 = tid / M, out_m0 = tid - out_f0 * M;                   // first output element of this thread
+    const int step_f = FEAT_THREADS / M, step_m = FEAT_THREADS - step_f * M;  // and the stride to its next one
 
     // samples of a tile: loaded into registers (all loads in flight together), mixed and
     // stored to `chunk` one phase later
@@ -468,30 +472,50 @@ frames_warp_kernel(const float *__restrict__ in_a, const float *__restrict__ in_
         if (vec) stage_store(); else stage_scalar(tile);
         __syncthreads();                      // chunk (and, first time, the tables) in place; sums of the last tile read
 
+        if (tile + 1 < n_tiles) {
+            // the next tile's stretch, 128 bytes per thread and array, into L2
+            const int nxt = (t0 + FT) * hop + (tid >> 1) * 32;
+            if (nxt < N) asm volatile("prefetch.global.L2 [%0];" ::"l"(((tid & 1) ? rb : ra) + nxt));
+        }
         const int f0 = 2 * warp;
         if (f0 < nf) {
             const bool have1 = f0 + 1 < nf;
             const float *c0 = chunk + f0 * hop;
             float2 v[2][8];
-            // butterfly b of the first pass is j = lane + 32 b: points j + 64 r
-#pragma unroll
-            for (int b = 0; b < 2; ++b) {
+            if (pairs) {
+                // First pass on butterflies j = 2 lane and 2 lane + 1 (points j + 64 r): adjacent
+                // samples, one 64-bit load each from the window table and the two frames.  A point
+                // beyond the window reads the window's last pair instead (its weight is zero).
 #pragma unroll
                 for (int r = 0; r < 8; ++r) {
-                    const int n = lane + 32 * (2 * r + b);
-                    float a = 0.f, bb = 0.f;
-                    if (n < win) {
-                        const float wn = win_s[n];
-                        a = wn * c0[n];
-                        if (have1) bb = wn * c0[hop + n];
+                    const int n = 2 * lane + 64 * r;
+                    const int nc = min(n, win - 2);
+                    const float2 wn = *reinterpret_cast<const float2 *>(win_s + n);
+                    const float2 a = *reinterpret_cast<const float2 *>(c0 + nc);
+                    const float2 bb = *reinterpret_cast<const float2 *>(c0 + hop + nc);
+                    v[0][r] = make_float2(wn.x * a.x, wn.x * bb.x);
+                    v[1][r] = make_float2(wn.y * a.y, wn.y * bb.y);
+                }
+            } else {
+#pragma unroll
+                for (int b = 0; b < 2; ++b) {
+#pragma unroll
+                    for (int r = 0; r < 8; ++r) {
+                        const int n = 2 * lane + b + 64 * r;
+                        float a = 0.f, bb = 0.f;
+                        if (n < win) {
+                            const float wn = win_s[n];
+                            a = wn * c0[n];
+                            if (have1) bb = wn * c0[hop + n];
+                        }
+                        v[b][r] = make_float2(a, bb);
                     }
-                    v[b][r] = make_float2(a, bb);
                 }
             }
             Dft<8>::run(v[0]);
             Dft<8>::run(v[1]);
-            scatter8<1>(v[0], xb, lane);
-            scatter8<1>(v[1], xb, lane + 32);
+            scatter8<1>(v[0], xb, 2 * lane);
+            scatter8<1>(v[1], xb, 2 * lane + 1);
             __syncwarp();
             gather<K, 16, 8, 1>(v, xb, lane);
             __syncwarp();
@@ -551,34 +575,58 @@ frames_warp_kernel(const float *__restrict__ in_a, const float *__restrict__ in_
         __syncthreads();                      // power spectra of the tile in place; chunk and the buffers are free
         if (vec && tile + 1 < n_tiles) stage_load(tile + 1);
 
-        // Filterbank with the frames of the tile over the lanes, two edge intervals per
-        // warp step: the bins of interval j give its rising sum (band j) and its falling
-        // sum (band j-1).
+        // Filterbank with the frames of the tile over the lanes, two adjacent edge
+        // intervals per warp step: the bins of interval j give its rising sum (band j) and
+        // its falling sum (band j-1).  Intervals widen with frequency, so the pairs are
+        // dealt to the warps from the widest down, back and forth, which evens out the
+        // bins each warp walks.
         {
             const int f = lane & (FT - 1), sub = lane / FT;
-            constexpr int BPW = 32 / FT;
-            for (int jb = warp * BPW; jb <= M; jb += WARPS * BPW) {
-                const int j = jb + sub;
-                if (j <= M && f < nf) {
+            static_assert(FT == 16, "two intervals per warp step");
+            const int npairs = (M + 2) / 2;                  // intervals 0 .. M in pairs (2q, 2q+1)
+            for (int st = 0; st * WARPS < npairs; ++st) {
+                const int q = npairs - 1 - (st * WARPS + ((st & 1) ? WARPS - 1 - warp : warp));
+                const int j = 2 * q + sub;
+                if (q >= 0 && j <= M && f < nf) {
                     const float *p = ptile + f * NBP;
-                    float u = 0.f, d = 0.f;
+                    float u0 = 0.f, d0 = 0.f, u1 = 0.f, d1 = 0.f;
+                    int k = mst[j];
                     const int k1 = mst[j + 1];
-                    for (int k = mst[j]; k < k1; ++k) {
-                        const float2 w = mw[k];
-                        const float pk = p[k];
-                        u = fmaf(w.x, pk, u);
-                        d = fmaf(w.y, pk, d);
+                    for (; k + 1 < k1; k += 2) {
+                        const float2 wa = mw[k], wb = mw[k + 1];
+                        const float pa = p[k], pb = p[k + 1];
+                        u0 = fmaf(wa.x, pa, u0);
+                        d0 = fmaf(wa.y, pa, d0);
+                        u1 = fmaf(wb.x, pb, u1);
+                        d1 = fmaf(wb.y, pb, d1);
                     }
-                    up_s[f * (M + 1) + j] = u;
-                    dn_s[f * (M + 1) + j] = d;
+                    if (k < k1) {
+                        const float2 wa = mw[k];
+                        const float pa = p[k];
+                        u0 = fmaf(wa.x, pa, u0);
+                        d0 = fmaf(wa.y, pa, d0);
+                    }
+                    up_s[f * (M + 1) + j] = u0 + u1;
+                    dn_s[f * (M + 1) + j] = d0 + d1;
                 }
             }
         }
         __syncthreads();                      // interval sums in place
         float *orow = orun + (int64_t)tile * FT * M;
-        for (int i = tid; i < nf * M; i += FEAT_THREADS) {
-            const int ff = i / M, m = i - ff * M;
-            orow[i] = compress(up_s[ff * (M + 1) + m] + dn_s[ff * (M + 1) + m + 1], floor_v, comp);
+        {
+            // element i = frame * M + band, walked without a division
+            int ff = out_f0, m = out_m0;
+            for (int i = tid; i < nf * M; i += FEAT_THREADS) {
+                const float e = fmaxf(up_s[ff * (M + 1) + m] + dn_s[ff * (M + 1) + m + 1], floor_v);
+                const float l = __logf(e);
+                orow[i] = comp == AUG_COMPRESS_LOG ? l : __expf(l * (1.f / 15.f));
+                ff += step_f;
+                m += step_m;
+                if (m >= M) {
+                    m -= M;
+                    ++ff;
+                }
+            }
         }
     }
 }
