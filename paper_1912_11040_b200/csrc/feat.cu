@@ -370,9 +370,30 @@ __device__ __forceinline__ void power_pair(float2 z, float2 q, float &pa, float 
 
 __host__ __device__ constexpr int chunk_floats(int win, int hop) { return ((FT - 1) * hop + win + 3) & ~3; }
 __host__ __device__ constexpr size_t smem_bytes(int win, int hop, int M) {
-    return sizeof(float2) * WARPS * XB + sizeof(float) * FT * NBP + sizeof(float) * chunk_floats(win, hop) +
-           sizeof(float) * K + sizeof(float2) * (NBP + 1) + sizeof(int) * (M + 2);
+    return sizeof(float2) * WARPS * XB + 3 * sizeof(float) * chunk_floats(win, hop) + sizeof(float) * K +
+           sizeof(float2) * (NBP + 1) + sizeof(int) * (M + 2);
 }
+
+// Once a warp's transforms are done its exchange buffer (2 XB floats) holds the two
+// power spectra of its frame pair and, behind them, the pair's interval sums.  Rows
+// start at different banks so that the frames of a tile can be read side by side.
+constexpr int ROW_SPAN = 2 * XB;                   // floats of a warp's buffer
+constexpr int SUMS_OFF = 2 * NBP + 2 * WARPS;      // floats before the sums of a pair
+__device__ __forceinline__ int power_row(int f) { return (f >> 1) * ROW_SPAN + (f & 1) * NBP + (f >> 1) * 2; }
+// sums of frame f: [rising, falling][M + 1]
+__device__ __forceinline__ int sums_row(int f, int M) {
+    return (f >> 1) * ROW_SPAN + SUMS_OFF + (f >> 1) * 4 + (f & 1) * 2 * (M + 1);
+}
+static_assert(SUMS_OFF + 4 * WARPS + 4 * (aug::MAX_MEL + 1) <= ROW_SPAN, "sums fit behind the power rows");
+
+// 16 bytes global -> shared without passing through registers; bytes = 0 stores zeros.
+__device__ __forceinline__ void copy16_async(float *dst_smem, const float *src, int bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(
+                     (unsigned)__cvta_generic_to_shared(dst_smem)),
+                 "l"(src), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void copies_done() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 
 template <int TILES>
 __global__ void __launch_bounds__(FEAT_THREADS, FEAT_MINB)
@@ -383,10 +404,12 @@ frames_warp_kernel(const float *__restrict__ in_a, const float *__restrict__ in_
                    float pad_v, int comp, float *__restrict__ out, int *__restrict__ counts, int n_cap) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int chunk_cap = chunk_floats(win, hop);
-    float2 *xb_all = reinterpret_cast<float2 *>(smem_raw);                   // [WARPS][XB]; later the interval sums
-    float *ptile = reinterpret_cast<float *>(xb_all + WARPS * XB);           // [FT][NBP]
-    float *chunk = ptile + FT * NBP;                                         // [chunk_cap]
-    float *win_s = chunk + chunk_cap;                                        // [K] Hann, zero beyond win
+    float2 *xb_all = reinterpret_cast<float2 *>(smem_raw);                   // [WARPS][XB]; later powers and sums
+    float *prow = reinterpret_cast<float *>(xb_all);
+    float *chunk = reinterpret_cast<float *>(xb_all + WARPS * XB);           // [chunk_cap] y_s + g v of the tile
+    float *raw_a = chunk + chunk_cap;                                        // [chunk_cap] y_s of the next tile
+    float *raw_b = raw_a + chunk_cap;                                        // [chunk_cap] v of the next tile
+    float *win_s = raw_b + chunk_cap;                                        // [K] Hann, zero beyond win
     float2 *mw = reinterpret_cast<float2 *>(win_s + K);                      // [NBP + 1] (up, down)
     int *mst = reinterpret_cast<int *>(mw + NBP + 1);                        // [M + 2]
 
@@ -426,36 +449,41 @@ frames_warp_kernel(const float *__restrict__ in_a, const float *__restrict__ in_
     twiddle_powers<8>(w3b, __ldg(&tw[tw_index(K, j1)]));
     const float2 w2_1 = __ldg(&tw[tw_index(64, lane & 7)]);
     float2 *xb = xb_all + warp * XB;
-    float *up_s = reinterpret_cast<float *>(xb_all);         // [FT][M + 1] rising sums (transforms are done)
-    float *dn_s = up_s + FT * (M + 1);                       // [FT][M + 1] falling sums
     const int n_tiles = min(TILES, (nfr + FT - 1) / FT);
     const int out_f0 = tid / M, out_m0 = tid - out_f0 * M;                   // first output element of this thread
     const int step_f = FEAT_THREADS / M, step_m = FEAT_THREADS - step_f * M;  // and the stride to its next one
 
-    // samples of a tile: loaded into registers (all loads in flight together), mixed and
-    // stored to `chunk` one phase later
-    float4 xa[SV], xv[SV];
-    auto stage_load = [&](int tile) {
+    // Samples of a tile travel global -> shared asynchronously, one tile ahead: a thread
+    // copies the 16-byte groups i = 4 (tid + 256 u) of y_s and v into raw_a / raw_b, and
+    // one tile later mixes the same groups into `chunk`, so the raw slots are private to
+    // the thread and need no barrier; groups beyond the tile's stretch are zero-filled.
+    auto stage_issue = [&](int tile) {
         const int s0 = (run0 + tile * FT) * hop;
         const int ns = (min(FT, T - (run0 + tile * FT)) - 1) * hop + win;
 #pragma unroll
         for (int u = 0; u < SV; ++u) {
             const int i = (tid + u * FEAT_THREADS) * 4;
-            xa[u] = xv[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (i < ns) {      // rows are allocated up to a multiple of 4 floats: whole groups can be read
-                xa[u] = __ldg(reinterpret_cast<const float4 *>(ra + s0 + i));
-                if (g != 0.f) xv[u] = __ldg(reinterpret_cast<const float4 *>(rb + s0 + i));
+            if (i < chunk_cap) {
+                // rows are allocated up to a multiple of 4 floats: whole groups can be read
+                const int ok = i < ns ? 16 : 0;
+                const int isrc = ok ? s0 + i : 0;
+                copy16_async(raw_a + i, ra + isrc, ok);
+                if (g != 0.f) copy16_async(raw_b + i, rb + isrc, ok);
             }
         }
     };
-    auto stage_store = [&]() {
+    auto stage_mix = [&]() {
 #pragma unroll
         for (int u = 0; u < SV; ++u) {
             const int i = (tid + u * FEAT_THREADS) * 4;
-            if (i < chunk_cap)
-                *reinterpret_cast<float4 *>(chunk + i) =
-                    make_float4(fmaf(g, xv[u].x, xa[u].x), fmaf(g, xv[u].y, xa[u].y),
-                                fmaf(g, xv[u].z, xa[u].z), fmaf(g, xv[u].w, xa[u].w));
+            if (i < chunk_cap) {
+                float4 x = *reinterpret_cast<const float4 *>(raw_a + i);
+                if (g != 0.f) {
+                    const float4 y = *reinterpret_cast<const float4 *>(raw_b + i);
+                    x = make_float4(fmaf(g, y.x, x.x), fmaf(g, y.y, x.y), fmaf(g, y.z, x.z), fmaf(g, y.w, x.w));
+                }
+                *reinterpret_cast<float4 *>(chunk + i) = x;
+            }
         }
     };
     auto stage_scalar = [&](int tile) {
@@ -463,20 +491,22 @@ frames_warp_kernel(const float *__restrict__ in_a, const float *__restrict__ in_
         const int ns = (min(FT, T - (run0 + tile * FT)) - 1) * hop + win;
         for (int i = tid; i < ns; i += FEAT_THREADS)
             chunk[i] = g != 0.f ? fmaf(g, rb[s0 + i], ra[s0 + i]) : ra[s0 + i];
+        for (int i = ns + tid; i < chunk_cap; i += FEAT_THREADS) chunk[i] = 0.f;
     };
-    if (vec) stage_load(0);
+    if (vec) stage_issue(0);
 
     for (int tile = 0; tile < n_tiles; ++tile) {
         const int t0 = run0 + tile * FT;
         const int nf = min(FT, T - t0);
-        if (vec) stage_store(); else stage_scalar(tile);
+        if (vec) {
+            copies_done();
+            stage_mix();
+            if (tile + 1 < n_tiles) stage_issue(tile + 1);
+        } else {
+            stage_scalar(tile);
+        }
         __syncthreads();                      // chunk (and, first time, the tables) in place; sums of the last tile read
 
-        if (tile + 1 < n_tiles) {
-            // the next tile's stretch, 128 bytes per thread and array, into L2
-            const int nxt = (t0 + FT) * hop + (tid >> 1) * 32;
-            if (nxt < N) asm volatile("prefetch.global.L2 [%0];" ::"l"(((tid & 1) ? rb : ra) + nxt));
-        }
         const int f0 = 2 * warp;
         if (f0 < nf) {
             const bool have1 = f0 + 1 < nf;
@@ -552,7 +582,8 @@ frames_warp_kernel(const float *__restrict__ in_a, const float *__restrict__ in_
             // Bin k pairs with bin 512 - k: for j0 + 64 r that is output 7 - r of the other
             // butterfly (lane 0: butterfly 0 pairs with itself, 64 r with 64 (8 - r), and so
             // does butterfly 32).  Only bins up to 256 are kept.
-            float *p0 = ptile + f0 * NBP, *p1 = p0 + NBP;
+            __syncwarp();                     // every lane has its last-pass inputs: the buffer is free
+            float *p0 = prow + power_row(f0), *p1 = prow + power_row(f0 + 1);
 #pragma unroll
             for (int r = 0; r < 4; ++r) {
                 const float2 qa = lane ? v[1][7 - r] : v[0][(8 - r) & 7];
@@ -572,8 +603,7 @@ frames_warp_kernel(const float *__restrict__ in_a, const float *__restrict__ in_
                 if (have1) p1[K / 2] = pb;
             }
         }
-        __syncthreads();                      // power spectra of the tile in place; chunk and the buffers are free
-        if (vec && tile + 1 < n_tiles) stage_load(tile + 1);
+        __syncthreads();                      // power spectra of the tile in place
 
         // Filterbank with the frames of the tile over the lanes, two adjacent edge
         // intervals per warp step: the bins of interval j give its rising sum (band j) and
@@ -588,7 +618,7 @@ frames_warp_kernel(const float *__restrict__ in_a, const float *__restrict__ in_
                 const int q = npairs - 1 - (st * WARPS + ((st & 1) ? WARPS - 1 - warp : warp));
                 const int j = 2 * q + sub;
                 if (q >= 0 && j <= M && f < nf) {
-                    const float *p = ptile + f * NBP;
+                    const float *p = prow + power_row(f);
                     float u0 = 0.f, d0 = 0.f, u1 = 0.f, d1 = 0.f;
                     int k = mst[j];
                     const int k1 = mst[j + 1];
@@ -606,8 +636,9 @@ frames_warp_kernel(const float *__restrict__ in_a, const float *__restrict__ in_
                         u0 = fmaf(wa.x, pa, u0);
                         d0 = fmaf(wa.y, pa, d0);
                     }
-                    up_s[f * (M + 1) + j] = u0 + u1;
-                    dn_s[f * (M + 1) + j] = d0 + d1;
+                    float *sm = prow + sums_row(f, M);
+                    sm[j] = u0 + u1;
+                    sm[M + 1 + j] = d0 + d1;
                 }
             }
         }
@@ -617,7 +648,8 @@ frames_warp_kernel(const float *__restrict__ in_a, const float *__restrict__ in_
             // element i = frame * M + band, walked without a division
             int ff = out_f0, m = out_m0;
             for (int i = tid; i < nf * M; i += FEAT_THREADS) {
-                const float e = fmaxf(up_s[ff * (M + 1) + m] + dn_s[ff * (M + 1) + m + 1], floor_v);
+                const float *sm = prow + sums_row(ff, M);
+                const float e = fmaxf(sm[m] + sm[M + 1 + m + 1], floor_v);
                 const float l = __logf(e);
                 orow[i] = comp == AUG_COMPRESS_LOG ? l : __expf(l * (1.f / 15.f));
                 ff += step_f;
