@@ -468,10 +468,11 @@ __device__ __forceinline__ void load_segment4(float2 (*va)[E], float2 (*vb)[E],
 // Passes two and three of both half transforms, shared by the forward and the
 // inverse direction (a real call: the kernel's instruction footprint matters).
 // On entry A is complete and visible and B at most one barrier away from it.
+// Returns with B written but not yet synchronised: the caller's barrier finishes it
+// (loads that do not depend on the transform go in front of that barrier).
 __device__ __noinline__ void fft2x4096_tail(float2 *A, float2 *B, int t, const float2 *__restrict__ tw) {
     pass_pair<N2, E, 16, 16, 1>(A, B, t, tw, CtaSync());
     pass_pair<N2, E, 16, 256, 16>(A, B, t, tw, CtaSync());
-    __syncthreads();
 }
 
 // Both half transforms of a segment held in registers; on return A and B hold the
@@ -483,6 +484,7 @@ __device__ __forceinline__ void fft2x4096_from_regs(float2 (*va)[E], float2 (*vb
     __syncthreads();
     fft2x4096_tail(A, B, t, tw);
 }
+// (both variants leave the closing barrier to the caller)
 
 __device__ __forceinline__ void fft2x4096_in_place(float2 *A, float2 *B, int t,
                                                    const float2 *__restrict__ tw) {
@@ -591,6 +593,7 @@ rir_spectra2_kernel(const float *__restrict__ rir, const AugUttParams *__restric
             vb[0][r] = make_float2(z.z, z.w);
         }
         fft2x4096_from_regs(va, vb, A, Bf, t, tw);
+        __syncthreads();
     }
 #pragma unroll
     for (int q = 0; q < NQ2; ++q) {
@@ -611,6 +614,25 @@ rir_spectra2_kernel(const float *__restrict__ rir, const AugUttParams *__restric
             out[N2 + k] = make_float2(x.pk.x * scale, x.pk.y * scale);
         }
     }
+}
+
+// What the spectral phase reads from global memory for slot k: the join and split
+// twiddles and the four response bins X[k], X[8192-k], X[4096-k], X[4096+k] pair with
+// (slot 0: the split twiddle of bin 2048 and bins 0/8192, 4096, 2048, 6144).
+struct SpecOps {
+    float2 w, u, h0, h1, h2, h3;
+};
+__device__ __forceinline__ SpecOps load_spec_ops(const float2 *__restrict__ H, const float2 *__restrict__ tw,
+                                                 int k) {
+    SpecOps o;
+    const bool z = k == 0;
+    o.w = __ldg(&tw[tw_index(NB2, k)]);
+    o.u = __ldg(&tw[z ? tw_index(F2, N2 / 2) : tw_index(F2, k)]);
+    o.h0 = __ldg(&H[k]);
+    o.h1 = __ldg(&H[z ? N2 : NB2 - k]);
+    o.h2 = __ldg(&H[z ? N2 / 2 : N2 - k]);
+    o.h3 = __ldg(&H[z ? N2 + N2 / 2 : N2 + k]);
+    return o;
 }
 
 // PARK: rows may have several noise sources (the context allows three or more
@@ -681,6 +703,9 @@ convolve_fused2_kernel(const float *__restrict__ speech, int64_t stride,
             fft2x4096_from_regs(va, vb, A, Bf, t, tw);
         }
         const float2 *H = hspec + ((int64_t)utt * S_max + s) * NB2;
+        // the first slot's operands are requested before the barrier that completes the transform
+        SpecOps nxt = load_spec_ops(H, tw, t);
+        __syncthreads();
         // what happens to this source's products: inverse-transformed right away (0),
         // parked for a later noise source (1: first one, 2: added to what is parked),
         // or joined by the parked sum before the inverse (3)
@@ -689,15 +714,16 @@ convolve_fused2_kernel(const float *__restrict__ speech, int64_t stride,
 #pragma unroll 2
         for (int q = 0; q < NQ2; ++q) {
             const int k = t + CT * q;
+            const SpecOps c = nxt;
+            if (q + 1 < NQ2) nxt = load_spec_ops(H, tw, k + CT);     // next slot's operands while this one is worked on
             float2 *pk = slot + (4 * q) * CT + t;      // this thread's four parked products, CT apart
             if (k == 0) {
-                const float2 uh = __ldg(&tw[tw_index(F2, N2 / 2)]);
+                const float2 uh = c.u;
                 Edge x4 = edge_forward(A[pad0(0)], Bf[pad0(0)], A[pad0(N2 / 2)], Bf[pad0(N2 / 2)], uh);
-                const float2 h0 = __ldg(&H[0]);
-                x4.dc = make_float2(x4.dc.x * h0.x, x4.dc.y * h0.y);
-                x4.mid = cmul(x4.mid, __ldg(&H[N2]));
-                x4.q1 = cmul(x4.q1, __ldg(&H[N2 / 2]));
-                x4.q3 = cmul(x4.q3, __ldg(&H[N2 + N2 / 2]));
+                x4.dc = make_float2(x4.dc.x * c.h0.x, x4.dc.y * c.h0.y);
+                x4.mid = cmul(x4.mid, c.h1);
+                x4.q1 = cmul(x4.q1, c.h2);
+                x4.q3 = cmul(x4.q3, c.h3);
                 if (PARK && mode >= 2) {
                     x4.dc = cadd(x4.dc, pk[0]);
                     x4.mid = cadd(x4.mid, pk[CT]);
@@ -713,12 +739,12 @@ convolve_fused2_kernel(const float *__restrict__ speech, int64_t stride,
                     edge_inverse(x4, uh, A[pad0(0)], Bf[pad0(0)], A[pad0(N2 / 2)], Bf[pad0(N2 / 2)]);
                 }
             } else {
-                const float2 w = __ldg(&tw[tw_index(NB2, k)]), u = __ldg(&tw[tw_index(F2, k)]);
+                const float2 w = c.w, u = c.u;
                 Quad x4 = quad_forward(A[pad0(k)], A[pad0(N2 - k)], Bf[pad0(k)], Bf[pad0(N2 - k)], w, u);
-                x4.k = cmul(x4.k, __ldg(&H[k]));
-                x4.nk = cmul(x4.nk, __ldg(&H[NB2 - k]));
-                x4.mk = cmul(x4.mk, __ldg(&H[N2 - k]));
-                x4.pk = cmul(x4.pk, __ldg(&H[N2 + k]));
+                x4.k = cmul(x4.k, c.h0);
+                x4.nk = cmul(x4.nk, c.h1);
+                x4.mk = cmul(x4.mk, c.h2);
+                x4.pk = cmul(x4.pk, c.h3);
                 if (PARK && mode >= 2) {
                     x4.k = cadd(x4.k, pk[0]);
                     x4.nk = cadd(x4.nk, pk[CT]);
@@ -743,6 +769,7 @@ convolve_fused2_kernel(const float *__restrict__ speech, int64_t stride,
         }
         __syncthreads();
         fft2x4096_in_place(A, Bf, t, tw);
+        __syncthreads();
 
         // The last `ob` outputs of the segment are this block: samples 4m, 4m+1 of the
         // segment are point m of A, samples 4m+2, 4m+3 point m of B.

@@ -224,6 +224,8 @@ __device__ __forceinline__ void pass_pair(float2 *a, float2 *b, int t, const flo
         float2 w[R];
         twiddle_powers<R>(w, __ldg(&tw[tw_index(NS * R, t & (NS - 1))]));
         // not unrolled: the second transform reuses the first one's instructions
+        // (building the powers after the first gather instead, to hide the table load,
+        // costs spills at this register budget and was slower)
 #pragma unroll 1
         for (int h = 0; h < 2; ++h) {
             float2 *s = h ? b : a;
