@@ -12,6 +12,9 @@ Steps and where the paper fixes them:
   reverb_mix         simulator block, Sections 1 / 2.3 (reverberate, add noise at an SNR)
   stft_power         feature block, Section 2.3
   vtlp_warp          Eq. 1 (bilinear frequency warp), exactly as printed
+  vtlp_resynth       the warp of Eq. 1 applied to the speech waveform with resynthesis
+                     (Section 2.3; 50 ms window of Section 4): this library's plain
+                     reading, fidelity to the authors' resynthesis PARITY UNPINNED
   mel_matrix/logmel  "mel filterbank energies", Section 2.3, with the warp of
                      Eq. 1 applied to the bin frequencies the triangles are
                      evaluated at; natural log (the paper's own power-law
@@ -179,6 +182,55 @@ def logmel(power, alpha, n_fft, n_mel, fs=16000.0, f_lo=0.0, f_hi=None, floor=1e
     raise ValueError(compression)
 
 
+# ---------------------------------------------------------------- waveform-domain VTLP
+def vtlp_unwarp(omega_out, alpha):
+    """The frequency whose content Eq. 1 moves to omega_out: the map of Eq. 1 is the
+    phase of a first-order all-pass with coefficient (1 - alpha); the all-pass with
+    the opposite coefficient undoes it."""
+    omega_out = np.asarray(omega_out, dtype=np.float64)
+    a = 1.0 - float(alpha)
+    return omega_out - 2.0 * np.arctan(a * np.sin(omega_out) / (1.0 + a * np.cos(omega_out)))
+
+
+def vtlp_resynth(x, alpha, win=800, n_fft=1024):
+    """Speech warped in the waveform domain (Section 2.3, the step before the
+    simulator; 50 ms window as in Section 4).  The paper prints only the frequency
+    map; this is the plain reading of "warp the spectrum and resynthesise":
+      frames of `win` samples every win/4, periodic Hann, the signal zero-padded by
+      win - win/4 samples in front so that every sample is covered by four frames;
+      DFT of n_fft points; the new spectrum at bin k is the old one at the frequency
+      Eq. 1 moves to bin k, taken by linear interpolation between the two nearest bins
+      (bins 0 and n_fft/2 stay); inverse DFT, first `win` samples, Hann again,
+      overlap-add, division by the summed squared windows.
+    Known defect of this reading: neighbouring frames of a steady tone no longer add
+    in phase, so the tone loses level.  alpha = 1 returns the input."""
+    x = np.asarray(x, dtype=np.float64)
+    N = x.size
+    hop = win // 4
+    front = win - hop
+    T = -(-(N + front) // hop) if N else 0
+    if T == 0:
+        return x.copy()
+    padded = np.zeros((T - 1) * hop + win)
+    padded[front:front + N] = x
+    w = 0.5 - 0.5 * np.cos(2.0 * np.pi * np.arange(win) / win)
+    nb = n_fft // 2 + 1
+    pos = vtlp_unwarp(2.0 * np.pi * np.arange(nb) / n_fft, alpha) * n_fft / (2.0 * np.pi)
+    pos[0], pos[-1] = 0.0, float(nb - 1)
+    k0 = np.minimum(np.floor(pos).astype(np.int64), nb - 2)
+    fr = pos - k0
+    acc = np.zeros_like(padded)
+    norm = np.zeros_like(padded)
+    for t in range(T):
+        seg = padded[t * hop: t * hop + win] * w
+        X = np.fft.rfft(seg, n_fft)
+        Y = (1.0 - fr) * X[k0] + fr * X[k0 + 1]
+        y = np.fft.irfft(Y, n_fft)[:win] * w
+        acc[t * hop: t * hop + win] += y
+        norm[t * hop: t * hop + win] += w * w
+    return acc[front:front + N] / norm[front:front + N]
+
+
 # ---------------------------------------------------------------- after the features
 def mfcc(feats, n_cep):
     """Orthonormal DCT-II of every row: c_i = s_i sum_m x[m] cos(pi i (m + 1/2)/M),
@@ -214,12 +266,17 @@ def utterance(speech, bank, row, cfg, compression="log"):
                              lattice=cfg.get("image_lattice", "total"))
             for s in range(n_src)]
     n = len(speech)
+    alpha_fb = float(row["alpha"])
+    if int(cfg.get("vtlp_win", 0)) > 0:
+        # the warp is applied to the speech waveform before the simulator; the filterbank stays unwarped
+        speech = vtlp_resynth(np.asarray(speech, dtype=np.float64), alpha_fb, int(cfg["vtlp_win"]))
+        alpha_fb = 1.0
     noises = [looped_noise(bank, row["noise_offset"][k], row["noise_len"][k], n)
               for k in range(n_src - 1)]
     wave, y_s, v, g = reverb_mix(np.asarray(speech, dtype=np.float64), rirs, noises,
                                  row["noise_weight"], row["snr_db"])
     power = stft_power(wave, int(cfg["win"]), int(cfg["hop"]), int(cfg["n_fft"]))
-    feats = logmel(power, float(row["alpha"]), int(cfg["n_fft"]), int(cfg["n_mel"]), fs,
+    feats = logmel(power, alpha_fb, int(cfg["n_fft"]), int(cfg["n_mel"]), fs,
                    float(cfg["f_lo"]), float(cfg["f_hi"]), float(cfg["log_floor"]), compression)
     return dict(rirs=rirs, y_s=y_s, v=v, g=g, wave=wave, power=power, feats=feats,
                 frames=power.shape[0])

@@ -45,6 +45,10 @@ PIN_CALLS = [
     lambda: pins.test_mel_partition_of_unity(0.9),
     lambda: pins.test_pure_tone_peaks_in_the_band_of_its_warped_frequency(0.8),
     pins.test_log_floor_and_power_law,
+    lambda: pins.test_unwarp_undoes_the_warp_of_eq1(0.85),
+    lambda: pins.test_resynthesis_without_warp_returns_the_input(801),
+    pins.test_resynthesis_is_linear,
+    lambda: pins.test_resynthesis_moves_a_tone_to_the_frequency_eq1_names(0.8),
 ]
 
 
@@ -132,7 +136,19 @@ def _mut_loop(bank, offset, length, n):
     return np.asarray(bank, dtype=np.float64)[idx]
 
 
+def _mut_unwarp_wrong_way(omega_out, alpha):
+    return oracle.vtlp_warp(omega_out, alpha)          # warps again instead of undoing
+
+
+def _mut_resynth_no_norm(x, alpha, win=800, n_fft=1024):
+    return 1.5 * _REAL_RESYNTH(x, alpha, win, n_fft)   # overlap-add not divided by the window sum
+
+
+_REAL_RESYNTH = oracle.vtlp_resynth
+
 PY_MUTATIONS = {
+    "spectrum moved the wrong way": ("vtlp_unwarp", _mut_unwarp_wrong_way),
+    "overlap-add without normalisation": ("vtlp_resynth", _mut_resynth_no_norm),
     "warp direction": ("vtlp_warp", _mut_warp_sign),
     "warp without the factor 2": ("vtlp_warp", _mut_warp_no_factor_two),
     "mel break frequency": ("hz_to_mel", _mut_mel),

@@ -396,6 +396,64 @@ def test_log_floor_and_power_law():
     np.testing.assert_allclose(pw, np.exp(lg / 15.0), rtol=1e-12)
 
 
+# ------------------------------------------------------------------ waveform-domain warp
+@pytest.mark.parametrize("alpha", [0.7, 0.85, 1.0, 1.2])
+def test_unwarp_undoes_the_warp_of_eq1(alpha):
+    w = np.linspace(0.0, np.pi, 301)
+    np.testing.assert_allclose(oracle.vtlp_unwarp(oracle.vtlp_warp(w, alpha), alpha), w, atol=1e-12)
+    # and it is the phase of the all-pass with the opposite coefficient
+    a = -(1.0 - alpha)
+    z = np.exp(1j * w)
+    np.testing.assert_allclose(oracle.vtlp_unwarp(w, alpha), np.unwrap(np.angle((z - a) / (1.0 - a * z))),
+                               atol=1e-12)
+
+
+@pytest.mark.parametrize("n", [1, 199, 200, 801, 5000])
+def test_resynthesis_without_warp_returns_the_input(n):
+    x = np.random.default_rng(n).standard_normal(n)
+    np.testing.assert_allclose(oracle.vtlp_resynth(x, 1.0), x, atol=1e-12)
+    np.testing.assert_allclose(oracle.vtlp_resynth(x, 1.0, win=400, n_fft=512), x, atol=1e-12)
+
+
+def test_resynthesis_is_linear():
+    rng = np.random.default_rng(4)
+    x1, x2 = rng.standard_normal(3000), rng.standard_normal(3000)
+    lhs = oracle.vtlp_resynth(2.5 * x1 - 0.75 * x2, 0.87)
+    rhs = 2.5 * oracle.vtlp_resynth(x1, 0.87) - 0.75 * oracle.vtlp_resynth(x2, 0.87)
+    np.testing.assert_allclose(lhs, rhs, atol=1e-12)
+
+
+@pytest.mark.parametrize("alpha", [0.8, 0.9, 1.1, 1.2])
+def test_resynthesis_moves_a_tone_to_the_frequency_eq1_names(alpha):
+    # a steady tone comes out near the warped frequency (within four bins of the 1024-point
+    # transform: frames no longer add in phase, which smears the line and costs level, the
+    # known weakness of warping frame by frame) and on the right side of where it started
+    f0 = 1500.0
+    y = oracle.vtlp_resynth(np.cos(2 * np.pi * f0 / FS * np.arange(16000)), alpha)
+    S = np.abs(np.fft.rfft(y[4000:12192] * np.hanning(8192)))
+    f_peak = np.argmax(S) * FS / 8192
+    a = 1.0 - alpha
+    z = np.exp(2j * np.pi * f0 / FS)
+    f_warp = np.angle((z - a) / (1.0 - a * z)) * FS / (2 * np.pi)
+    assert abs(f_peak - f_warp) <= 4 * FS / 1024
+    assert (f_peak > f0 + 200) == (alpha < 1) and (f_peak < f0 - 200) == (alpha > 1)
+    assert 0.2 < np.sqrt(np.mean(y[2000:14000] ** 2)) / np.sqrt(0.5) < 1.0
+
+
+def test_whole_path_with_the_waveform_warp_leaves_the_filterbank_unwarped():
+    from paper_1912_11040_b200 import synth
+    x = synth.speech_like(np.random.default_rng(8), 6000)
+    row = np.zeros(1, dtype=synth.UTT_DTYPE)[0]
+    row["room"], row["mic"], row["src_pos"][0] = (50, 8, 4), (2, 3, 1.5), (2 + 42.875, 3, 1.5)
+    row["n_src"], row["order"], row["alpha"], row["snr_db"] = 1, 0, 0.85, 10.0
+    cfg = dict(synth._COMMON, rir_taps=4096, max_order=0, vtlp_win=800)
+    out = oracle.utterance(x, np.zeros(16), row, cfg)
+    xw = oracle.vtlp_resynth(x, float(np.float32(0.85)))      # the table stores the factor in fp32
+    np.testing.assert_allclose(out["wave"][2000:], xw[:-2000] / 42.875, atol=1e-13)
+    ref = oracle.logmel(oracle.stft_power(out["wave"], 400, 160, 512), 1.0, 512, 40, floor=cfg["log_floor"])
+    np.testing.assert_allclose(out["feats"], ref, atol=1e-9)
+
+
 # ------------------------------------------------------------------ whole path
 def test_delta_rir_path_returns_the_input_features():
     # beta = 0 and a source 42.875 m = 343/8 m away (exact in fp32, as the table
