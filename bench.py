@@ -368,7 +368,9 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     # every rank runs the same kind of job on its own draw of the workload
-    w = synth.make_workload(args.workload, seed=rank, batch=args.batch)
+    w = synth.make_workload(args.workload, seed=rank, batch=args.batch, noise_align=args.noise_align)
+    if args.vtlp_win:
+        w.cfg["vtlp_win"] = args.vtlp_win          # warp the speech waveform instead of the filterbank
     cfg = binding.make_config(w.cfg, w.B, w.stride, host_staging=True, max_bank_samples=w.bank.size)
     ctx = binding.AugContext(cfg)
     speech = torch.from_numpy(w.speech).cuda()
@@ -404,6 +406,32 @@ def run_ours(args):
     clocks = sampler.stop()
     ms_total = e0.elapsed_time(e1)
     launches = ctx.aug_launch_count() - launches0
+    # ---- the same audio with noise stretches that start and end anywhere (the default
+    # recipe hands out stretches on multiples of four samples)
+    ms_unaligned = None
+    if args.noise_align > 1 and not args.skip_e2e:
+        table_un = binding.table_to_device(
+            synth.redraw_noise_stretches(w.table, w.lengths, w.bank.size, seed=rank, noise_align=1))
+        rc_un, bad_un = binding.aug_validate_params(cfg, synth.redraw_noise_stretches(
+            w.table, w.lengths, w.bank.size, seed=rank, noise_align=1), w.bank.size)
+        assert rc_un == 0, f"unaligned table row {bad_un} invalid"
+
+        def step_un():
+            ctx.aug_pipeline(speech, w.stride, lengths, w.lengths, bank, w.bank.size, table_un, w.B,
+                             feats, T_max, counts)
+
+        for _ in range(3):
+            step_un()
+        barrier()
+        u0, u1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        u0.record()
+        for _ in range(args.steps):
+            step_un()
+        u1.record()
+        barrier()
+        ms_unaligned = u0.elapsed_time(u1) / args.steps
+        assert ctx.aug_last_status() == (-1, 0)
+
     # ---- per-stage times: the same steps again with an event pair around every stage
     ctx.aug_enable_stage_timing(True)
     for _ in range(min(args.steps, 100)):
@@ -520,7 +548,7 @@ def run_ours(args):
             "warmup": max(args.warmup, 3), "ms_per_step": ms_total / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
             "data": "synthetic",
-            "config": {"workload": workload_label(args.workload), "batch": w.B,
+            "config": {"workload": workload_label(args.workload), "batch": w.B, "noise_align": args.noise_align, "vtlp_win": args.vtlp_win,
                        "audio_seconds_per_step": w.audio_seconds, "parallelism": f"replicas x{world}",
                        "l2": "inputs larger than L2 (speech + noise bank "
                              f"{(speech.numel() + bank.numel()) * 4 / 1e6:.0f} MB per step)"},
@@ -531,6 +559,11 @@ def run_ours(args):
             "roofline": roofline,
             "cpu_baseline": {"value": cpu_val, "unit": UNIT, "cores": cores, "kind": "oracle",
                              "sample": cpu_sample}}
+    if ms_unaligned is not None:
+        line["noise_unaligned"] = {"ms_per_step": ms_unaligned,
+                                   "value": w.audio_seconds * world / (ms_unaligned * 1e-3), "unit": UNIT,
+                                   "note": "same audio, noise stretches at any offset and length (rank 0's "
+                                           "own time); the headline uses stretches on multiples of 4 samples"}
     if dt_res > 0:
         line["e2e_resident_bank"] = {"value": audio_total * e2e_steps / dt_res, "unit": UNIT,
                                      "h2d_bytes_per_step": h2d_res, "d2h_bytes_per_step": d2h,
@@ -558,6 +591,11 @@ def main():
                     help="seconds of wall time given to the CPU-checker baseline")
     ap.add_argument("--cpu-fast-utts", type=int, default=64,
                     help="utterances given to the numpy/scipy CPU pipeline (0 = skip)")
+    ap.add_argument("--noise-align", type=int, default=4, choices=[1, 4],
+                    help="noise stretches start and end on multiples of this many samples (1 = anywhere)")
+    ap.add_argument("--vtlp-win", type=int, default=0,
+                    help="apply the warp to the speech waveform with this window (800 = 50 ms) instead of "
+                         "inside the filterbank")
     ap.add_argument("--batch", type=int, default=None,
                     help="profiling runs: fewer utterances than the workload's own batch")
     ap.add_argument("--skip-e2e", action="store_true",

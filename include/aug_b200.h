@@ -78,6 +78,11 @@ typedef struct {
     int32_t host_staging;    /* non-zero: also allocate device staging for aug_pipeline_host */
     int32_t image_lattice;   /* AugLattice */
     int64_t max_bank_samples; /* capacity of the staged noise bank (host_staging only) */
+    int32_t vtlp_win;        /* 0: the warp of Eq. 1 acts inside the mel filterbank (default).
+                                > 0: it is applied to the speech waveform before the simulator,
+                                with this window (samples; a multiple of 4, at most 1024; 800 is
+                                the 50 ms of Section 4) and the filterbank stays unwarped */
+    int32_t reserved_;       /* keeps the struct a multiple of 8 bytes; set to 0 */
 } AugConfig;
 
 /*
@@ -170,6 +175,22 @@ int aug_destroy(AugCtx *ctx);
  * short of a launch failure).  A rejected utterance gets zero impulse
  * responses / silent output; nothing faults.  The word is cleared by the read. */
 int aug_last_status(AugCtx *ctx, int *utt_host, int *reason_host);
+
+/* -------------------------------------------------------------- before step 1 (optional)
+ * VTLP on the waveform with resynthesis (Section 2.3: the warp of Eq. 1 is applied to
+ * the speech before the acoustic simulator, so that noise and reverberation are not
+ * warped; Section 4 finds a 50 ms window best).  The paper prints only the frequency
+ * map; what is computed here: frames of vtlp_win samples every vtlp_win/4, periodic
+ * Hann, the utterance zero-padded by 3 vtlp_win/4 in front; 1024-point DFT; the
+ * spectrum at bin k becomes the old spectrum at the frequency that Eq. 1 moves to
+ * bin k, by linear interpolation between the two nearest bins; inverse DFT, first
+ * vtlp_win samples, Hann again, overlap-add, division by the summed squared windows.
+ * alpha = 1 returns the input.
+ *   speech_dev [B][stride] -> warped_dev [B][out_stride], samples [0, lengths[b]) written
+ * Needs a context created with vtlp_win > 0 (AUG_EINVAL otherwise).  aug_pipeline of
+ * such a context runs this on the speech first and builds the filterbank unwarped. */
+int aug_vtlp_resynth(AugCtx *ctx, const float *speech_dev, int64_t stride, const int *lengths_dev,
+                     const AugUttParams *table_dev, int B, float *warped_dev, int64_t out_stride);
 
 /* -------------------------------------------------------------- step 1
  * Room impulse responses by the image-source method (simulator block, Sections

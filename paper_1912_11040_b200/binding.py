@@ -24,7 +24,7 @@ EXPORTS = ["aug_strerror", "aug_frame_count", "aug_workspace_bytes", "aug_valida
            "aug_reverb_mix", "feat_stft_power", "feat_vtlp_logmel", "aug_pipeline",
            "aug_pipeline_host", "aug_enable_stage_timing", "aug_stage_times", "aug_launch_count",
            "aug_measure_fp32_peak", "feat_vtlp_logmel_noalloc", "aug_last_host_bytes", "aug_upload_noise_bank", "aug_hold_parking_slots", "aug_sample_params", "feat_mfcc", "feat_mean_var",
-           "aug_bucket_by_length"]
+           "aug_bucket_by_length", "aug_vtlp_resynth"]
 NOALLOC_MAX_BATCH = 256
 N_STAGES = 7
 STAGE_NAMES = ["rir_image", "rir_spectra", "mel_tables", "block_spectra", "convolve", "mix",
@@ -40,7 +40,8 @@ class AugConfig(ctypes.Structure):
                 ("log_floor", ctypes.c_float), ("pad_value", ctypes.c_float),
                 ("compression", ctypes.c_int32), ("max_batch", ctypes.c_int32),
                 ("max_samples", ctypes.c_int32), ("host_staging", ctypes.c_int32),
-                ("image_lattice", ctypes.c_int32), ("max_bank_samples", ctypes.c_int64)]
+                ("image_lattice", ctypes.c_int32), ("max_bank_samples", ctypes.c_int64),
+                ("vtlp_win", ctypes.c_int32), ("reserved_", ctypes.c_int32)]
 
 
 class AugDist(ctypes.Structure):
@@ -86,6 +87,8 @@ def lib() -> ctypes.CDLL:
         L.aug_destroy.argtypes = [vp]
         L.aug_last_status.restype = i32
         L.aug_last_status.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(i32)]
+        L.aug_vtlp_resynth.restype = i32
+        L.aug_vtlp_resynth.argtypes = [vp, vp, i64, vp, vp, i32, vp, i64]
         L.aug_rir_image_method.restype = i32
         L.aug_rir_image_method.argtypes = [vp, vp, i32, vp]
         L.aug_reverb_mix.restype = i32
@@ -146,7 +149,8 @@ def make_config(cfg: dict, max_batch: int, max_samples: int, *, compression: int
                      pad_value=float(cfg["pad_value"]), compression=int(compression),
                      max_batch=int(max_batch), max_samples=int(max_samples),
                      host_staging=int(bool(host_staging)), image_lattice=int(image_lattice),
-                     max_bank_samples=int(max_bank_samples))
+                     max_bank_samples=int(max_bank_samples), vtlp_win=int(cfg.get("vtlp_win", 0)),
+                     reserved_=0)
 
 
 def aug_workspace_bytes(config: AugConfig) -> int:
@@ -292,6 +296,12 @@ class AugContext:
         _check(lib().aug_last_host_bytes(self._h, ctypes.byref(a), ctypes.byref(b)),
                "aug_last_host_bytes")
         return int(a.value), int(b.value)
+
+    def aug_vtlp_resynth(self, speech_dev, stride, lengths_dev, table_dev, B, warped_dev, out_stride,
+                         check=True):
+        return self._ret(lib().aug_vtlp_resynth(self._h, _ptr(speech_dev), int(stride), _ptr(lengths_dev),
+                                                _ptr(table_dev), int(B), _ptr(warped_dev),
+                                                int(out_stride)), "aug_vtlp_resynth", check)
 
     def aug_rir_image_method(self, table_dev, B, rir_dev, check=True):
         return self._ret(lib().aug_rir_image_method(self._h, _ptr(table_dev), int(B),

@@ -5,7 +5,7 @@ import subprocess
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libaugb200.so")
-SOURCES = ["api.cu", "rir.cu", "conv.cu", "feat.cu", "peak.cu", "sample.cu", "post.cu"]
+SOURCES = ["api.cu", "rir.cu", "conv.cu", "feat.cu", "peak.cu", "sample.cu", "post.cu", "resynth.cu"]
 HEADERS = ["common.cuh", "fft.cuh", os.path.join("..", "..", "include", "aug_b200.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-shared", "-cudart", "static"]

@@ -72,6 +72,7 @@ int check_config(const AugConfig *c) {
     if (c->image_lattice != AUG_LATTICE_TOTAL && c->image_lattice != AUG_LATTICE_CUBE) return AUG_EINVAL;
     if (c->max_batch < 1 || c->max_batch > 65535 || c->max_samples < 1) return AUG_EINVAL;
     if (c->host_staging && c->max_bank_samples < 0) return AUG_EINVAL;
+    if (c->vtlp_win < 0 || c->vtlp_win > 1024 || (c->vtlp_win & 3)) return AUG_EINVAL;
     return AUG_OK;
 }
 
@@ -80,7 +81,7 @@ struct Layout {
     int64_t ws_stride;
     int64_t off_xspec, off_park, off_park_flags;
     int64_t off_tw, off_rir, off_hspec, off_ys, off_vv, off_energy, off_gain, off_melw, off_melstart,
-        off_status, off_st_speech, off_st_bank, off_st_table, off_st_lengths,
+        off_status, off_warped, off_st_speech, off_st_bank, off_st_table, off_st_lengths,
         off_st_feats, off_st_counts, total;
 };
 
@@ -110,6 +111,7 @@ Layout make_layout(const AugConfig &c) {
     l.off_melw = take(sizeof(aug::MelBin) * B * l.n_bins);
     l.off_melstart = take(sizeof(int) * B * (c.n_mel + 2));
     l.off_status = take(sizeof(int) * 2);
+    l.off_warped = c.vtlp_win > 0 ? take(sizeof(float) * B * l.ws_stride) : -1;
     if (c.host_staging) {
         l.off_st_speech = take(sizeof(float) * B * l.ws_stride);
         l.off_st_bank = take(sizeof(float) * (c.max_bank_samples > 0 ? c.max_bank_samples : 1));
@@ -241,6 +243,7 @@ int aug_create(AugCtx **out, const AugConfig *cfg, void *cuda_stream) {
     ctx->melw = reinterpret_cast<aug::MelBin *>(base + l.off_melw);
     ctx->melstart = reinterpret_cast<int *>(base + l.off_melstart);
     ctx->status = reinterpret_cast<int *>(base + l.off_status);
+    ctx->warped = l.off_warped >= 0 ? reinterpret_cast<float *>(base + l.off_warped) : nullptr;
     if (cfg->host_staging) {
         ctx->st_speech = reinterpret_cast<float *>(base + l.off_st_speech);
         ctx->st_bank = reinterpret_cast<float *>(base + l.off_st_bank);
@@ -328,6 +331,20 @@ int aug_last_status(AugCtx *ctx, int *utt, int *reason) {
     if (utt) *utt = st[0];
     if (reason) *reason = st[0] >= 0 ? st[1] : 0;
     return AUG_OK;
+}
+
+int aug_vtlp_resynth(AugCtx *ctx, const float *speech_dev, int64_t stride, const int *lengths_dev,
+                     const AugUttParams *table_dev, int B, float *warped_dev, int64_t out_stride) {
+    int rc = check_batch(ctx, B);
+    if (rc != AUG_OK) return rc;
+    if (ctx->cfg.vtlp_win <= 0) return AUG_EINVAL;
+    if (B == 0) return AUG_OK;
+    if (!speech_dev || !lengths_dev || !table_dev || !warped_dev || stride <= 0 || out_stride <= 0)
+        return AUG_EINVAL;
+    const int64_t cap = stride < out_stride ? stride : out_stride;
+    const int max_len = (int)(cap < ctx->cfg.max_samples ? cap : ctx->cfg.max_samples);
+    return launch_vtlp_resynth(ctx, speech_dev, stride, lengths_dev, table_dev, B, max_len, warped_dev,
+                               out_stride);
 }
 
 int aug_rir_image_method(AugCtx *ctx, const AugUttParams *table_dev, int B, float *rir_dev) {
@@ -423,7 +440,14 @@ int aug_pipeline(AugCtx *ctx, const float *speech_dev, int64_t speech_stride,
     if (rc == AUG_OK) rc = launch_mel_tables(ctx, table_dev, B, ss);
     t1(2, ss);
 
+    // waveform-domain warp first: the simulator then sees the warped speech (timed with stage 3)
     t0(3, sm);
+    if (rc == AUG_OK && ctx->warped) {
+        rc = launch_vtlp_resynth(ctx, speech_dev, speech_stride, lengths_dev, table_dev, B, max_len,
+                                 ctx->warped, ctx->ws_stride);
+        speech_dev = ctx->warped;
+        speech_stride = ctx->ws_stride;
+    }
     if (rc == AUG_OK)
         rc = launch_convolve_prepare(ctx, speech_dev, speech_stride, lengths_dev, noise_bank_dev,
                                      bank_len, table_dev, B, max_len);

@@ -63,6 +63,7 @@ struct AugCtx {
     float2 *park;          // [PARK_SMS * 3][8192] products of noise sources waiting for the last one; NULL if unused
     int *park_flags;       // [PARK_SMS * 3] 1 = slot taken
     int n_sm;              // multiprocessors with slots (PARK_SMS); CTAs on others sum in the time domain
+    float *warped;         // [max_batch][ws_stride] speech after the waveform warp; NULL unless cfg.vtlp_win
     float *ys;             // [max_batch][ws_stride]
     float *vv;             // [max_batch][ws_stride]
     double *energy;        // [max_batch][2]
@@ -130,6 +131,8 @@ int launch_convolve_finish(AugCtx *ctx, const float *speech, int64_t stride, con
 int launch_mix(AugCtx *ctx, const int *lengths, const AugUttParams *table, int B, int max_len,
                float *wave_out, int64_t out_stride);
 int launch_mel_tables(AugCtx *ctx, const AugUttParams *table, int B, cudaStream_t st);
+int launch_vtlp_resynth(AugCtx *ctx, const float *speech, int64_t stride, const int *lengths,
+                        const AugUttParams *table, int B, int max_len, float *out, int64_t out_stride);
 int launch_stft_power(AugCtx *ctx, const float *wave, int64_t stride, const int *lengths, int B,
                       float *power, int T_max, int *counts);
 int launch_logmel(AugCtx *ctx, const float *power, const int *counts, int B, int T_max,

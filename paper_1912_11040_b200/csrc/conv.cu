@@ -395,7 +395,7 @@ constexpr int NQ2 = N2 / 2 / CT;       // slot pairs per thread and buffer
 // base + 4 (t + 256 r) + {0,1} as point r of buffer A and + {2,3} as point r of B.
 __device__ __forceinline__ void load_segment4(float2 (*va)[E], float2 (*vb)[E],
                                               const float *__restrict__ x, bool looped, int nlen,
-                                              int base, int N, int t) {
+                                              int base, int N, int t, const float *xend) {
     if (!looped) {
 #pragma unroll
         for (int r = 0; r < E; ++r) {
@@ -440,13 +440,24 @@ __device__ __forceinline__ void load_segment4(float2 (*va)[E], float2 (*vb)[E],
         }
         return;
     }
+    // Any other stretch: a group of four that does not wrap is read as the aligned
+    // 128-bit word it starts in and, if it starts a samples into that word, the next
+    // word as well (a second round, so that the first loads are all in flight
+    // together; neighbouring threads bring that word into L1).  Groups that wrap, end
+    // with the utterance or would touch bytes past the bank are read sample by sample.
+    const int m0 = m;
+    const int room = (int)min((int64_t)0x7fffffff, (int64_t)(xend - x));   // samples from x to the end of the bank
+    const int a0 = (int)((reinterpret_cast<uintptr_t>(x) >> 2) & 3);       // where in a 128-bit word x starts
+    unsigned amask = 0;                  // 2 bits per group: a, where the second round is needed
 #pragma unroll
     for (int r = 0; r < E; ++r) {
         const int i0 = first + 4 * CT * r;
         float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
         if (i0 >= 0 && i0 < N) {
-            if (m + 3 < nlen && i0 + 3 < N) {
-                z = make_float4(x[m], x[m + 1], x[m + 2], x[m + 3]);
+            const int a = (a0 + m) & 3;
+            if (m + 3 < nlen && i0 + 3 < N && (a == 0 || m - a + 8 <= room)) {
+                z = __ldg(reinterpret_cast<const float4 *>(x + (m - a)));
+                amask |= (unsigned)a << (2 * r);
             } else {
                 int j = m;
                 z.x = x[j];
@@ -462,6 +473,24 @@ __device__ __forceinline__ void load_segment4(float2 (*va)[E], float2 (*vb)[E],
         vb[0][r] = make_float2(z.z, z.w);
         m += step;
         if (m >= nlen) m -= nlen;
+    }
+    if (__any_sync(0xffffffffu, amask != 0)) {
+        m = m0;
+#pragma unroll
+        for (int r = 0; r < E; ++r) {
+            const int a = (int)(amask >> (2 * r)) & 3;
+            if (a) {
+                const float4 q = __ldg(reinterpret_cast<const float4 *>(x + m - a + 4));
+                const float2 lo = va[0][r], hi = vb[0][r];
+                // samples a .. a+3 of the eight in (lo, hi, q)
+                va[0][r] = a == 1 ? make_float2(lo.y, hi.x) : a == 2 ? hi : make_float2(hi.y, q.x);
+                vb[0][r] = a == 1 ? make_float2(hi.y, q.x) : a == 2 ? make_float2(q.x, q.y) : make_float2(q.y, q.z);
+            }
+            m += step;
+            if (m >= nlen) m -= nlen;
+            // four second-round loads at a time: more in flight would not fit the registers
+            if ((r & 3) == 3) asm volatile("" ::: "memory");
+        }
     }
 }
 
@@ -699,7 +728,7 @@ convolve_fused2_kernel(const float *__restrict__ speech, int64_t stride,
         if (!source_of(row, s, speech + (int64_t)utt * stride, bank, bank_len, x, nlen)) continue;
         {
             float2 va[1][E], vb[1][E];
-            load_segment4(va, vb, x, s != 0, nlen, (b + 1) * ob - F2, N, t);
+            load_segment4(va, vb, x, s != 0, nlen, (b + 1) * ob - F2, N, t, bank + bank_len);
             fft2x4096_from_regs(va, vb, A, Bf, t, tw);
         }
         const float2 *H = hspec + ((int64_t)utt * S_max + s) * NB2;

@@ -31,10 +31,11 @@ __host__ __device__ __forceinline__ int frame_count(int n, int win, int hop) {
 // rounding), then the first bin of every interval.
 __global__ void __launch_bounds__(256)
 mel_tables_kernel(const AugUttParams *__restrict__ table, int K, int M, double fs, double f_lo,
-                  double f_hi, aug::MelBin *__restrict__ melw, int *__restrict__ melstart) {
+                  double f_hi, aug::MelBin *__restrict__ melw, int *__restrict__ melstart, int unwarped) {
     __shared__ int seg_s[513];
     const int utt = blockIdx.x, nb = K / 2 + 1;
-    const double a = 1.0 - (double)table[utt].alpha;
+    // (unwarped: the warp was already applied to the waveform)
+    const double a = unwarped ? 0.0 : 1.0 - (double)table[utt].alpha;
     const double PI = 3.14159265358979323846;
     const double e0 = 2595.0 * log10(1.0 + f_lo / 700.0);
     const double e1 = 2595.0 * log10(1.0 + f_hi / 700.0);
@@ -728,7 +729,7 @@ int launch_mel_tables(AugCtx *ctx, const AugUttParams *table, int B, cudaStream_
     const AugConfig &c = ctx->cfg;
     mel_tables_kernel<<<B, 256, 0, st>>>(table, c.n_fft, c.n_mel, (double)c.fs,
                                                   (double)c.f_lo, (double)c.f_hi, ctx->melw,
-                                                  ctx->melstart);
+                                                  ctx->melstart, c.vtlp_win > 0 ? 1 : 0);
     AUG_CUDA_OK(cudaGetLastError());
     ctx->launches++;
     return AUG_OK;
@@ -871,7 +872,7 @@ extern "C" int feat_vtlp_logmel_noalloc(const AugConfig *cfg, const float *power
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     const int nbp = cfg->n_fft / 2 + 1;
     mel_tables_kernel<<<B, 256, 0, st>>>(table_dev, cfg->n_fft, cfg->n_mel, (double)cfg->fs,
-                                         (double)cfg->f_lo, (double)cfg->f_hi, melw, melstart);
+                                         (double)cfg->f_lo, (double)cfg->f_hi, melw, melstart, 0);
     AUG_CUDA_OK(cudaGetLastError());
     const size_t smem = sizeof(aug::MelBin) * (nbp + 1) + sizeof(int) * (cfg->n_mel + 2);
     dim3 grid((T_max + 7) / 8, B);

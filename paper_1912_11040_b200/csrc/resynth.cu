@@ -1,0 +1,182 @@
+// Waveform-domain VTLP: the warp of Eq. 1 applied to the speech itself, with
+// resynthesis, before the simulator (Section 2.3; 50 ms window of Section 4).
+//
+// The paper prints only the frequency map.  The reading built here: frames of
+// `win` samples every win/4, periodic Hann, the utterance zero-padded by
+// win - win/4 samples in front; 1024-point DFT; the spectrum at bin k becomes the
+// old spectrum at the frequency that Eq. 1 moves to bin k (the all-pass with the
+// opposite coefficient), by linear interpolation between the two nearest bins;
+// inverse DFT, first `win` samples, Hann again, overlap-add, division by the sum
+// of the squared windows.
+//
+// Two frames ride through the transforms as the real and imaginary part of one
+// complex signal: interpolation is linear, so it acts on the packed spectrum Z
+// directly (bin k from Z around k0, bin K-k from Z around K-k0), and the inverse of
+// the packed spectrum returns the two frames in its real and imaginary part.
+// A CTA owns the output samples of HB hops and computes the HB + 3 frames that
+// cover them, so nothing is added across CTAs.
+#include "common.cuh"
+#include "fft.cuh"
+
+namespace {
+
+using namespace augfft;
+constexpr int K = 1024;
+constexpr int E = 16;                 // points per thread
+constexpr int GROUP = K / E;          // 64 threads per transform
+constexpr int NGROUP = 2;
+constexpr int RS_THREADS = GROUP * NGROUP;
+constexpr int HB = 8;                 // hops of output per CTA
+constexpr int NF = HB + 3;            // frames that cover them
+constexpr int XB = padded_points(K);
+
+__host__ __device__ constexpr size_t resynth_smem(int win) {
+    const int hop = win / 4;
+    return sizeof(float2) * 2 * NGROUP * XB + sizeof(float) * (size_t)((NF - 1) * hop + win) +
+           sizeof(float) * (size_t)NF * win + sizeof(float) * win + sizeof(float) * (K / 2 + 1) +
+           sizeof(int) * (K / 2 + 1);
+}
+
+__device__ __forceinline__ void fft1024_from_regs(float2 (*v)[E], float2 *s, int tg, const float2 *__restrict__ tw,
+                                                  GroupSync gsync) {
+    pass_from_regs<K, E, E, 1>(v, s, tg, tw);
+    gsync();
+    pass<K, E, 8, 16, 1>(s, tg, tw, gsync);
+    pass<K, E, 8, 128, 16>(s, tg, tw, gsync);
+}
+__device__ __forceinline__ void fft1024_in_place(float2 *s, int tg, const float2 *__restrict__ tw, GroupSync gsync) {
+    pass<K, E, E, 1, 0>(s, tg, tw, gsync);
+    pass<K, E, 8, 16, 1>(s, tg, tw, gsync);
+    pass<K, E, 8, 128, 16>(s, tg, tw, gsync);
+}
+
+__global__ void __launch_bounds__(RS_THREADS)
+vtlp_resynth_kernel(const float *__restrict__ speech, int64_t stride, const int *__restrict__ lengths,
+                    const AugUttParams *__restrict__ table, int win, const float2 *__restrict__ tw,
+                    float *__restrict__ out, int64_t out_stride, int n_cap) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int hop = win >> 2, front = win - hop;
+    float2 *zbuf = reinterpret_cast<float2 *>(smem_raw);            // [NGROUP][XB] forward transforms
+    float2 *wbuf = zbuf + NGROUP * XB;                              // [NGROUP][XB] warped spectra / inverse
+    float *xin = reinterpret_cast<float *>(wbuf + NGROUP * XB);     // [(NF-1) hop + win] padded input stretch
+    float *fout = xin + (NF - 1) * hop + win;                       // [NF][win] resynthesised, windowed frames
+    float *wn = fout + NF * win;                                    // [win] Hann
+    float *fr_s = wn + win;                                         // [K/2+1] interpolation fraction
+    int *k0_s = reinterpret_cast<int *>(fr_s + K / 2 + 1);          // [K/2+1] lower source bin
+
+    const int utt = blockIdx.y, tid = threadIdx.x, tg = tid & (GROUP - 1), grp = tid / GROUP;
+    const int N = min(max(lengths[utt], 0), n_cap);
+    if (N == 0) return;
+    const int T = (N + front + hop - 1) / hop;       // frames = hops that cover the padded utterance
+    const int t0 = blockIdx.x * HB;                  // first hop this CTA owns
+    if (t0 >= T) return;
+    const float *x = speech + (int64_t)utt * stride;
+    float *y = out + (int64_t)utt * out_stride;
+
+    // source position of every bin: the frequency Eq. 1 moves to bin k, in bins
+    {
+        const double a = 1.0 - (double)table[utt].alpha;
+        const double PI = 3.14159265358979323846;
+        for (int k = tid; k <= K / 2; k += RS_THREADS) {
+            const double om = 2.0 * PI * k / K;
+            double pos = (om - 2.0 * atan(a * sin(om) / (1.0 + a * cos(om)))) * K / (2.0 * PI);
+            if (k == 0) pos = 0.0;
+            if (k == K / 2) pos = (double)(K / 2);
+            int k0 = (int)floor(pos);
+            k0 = min(max(k0, 0), K / 2 - 1);
+            k0_s[k] = k0;
+            fr_s[k] = (float)(pos - (double)k0);
+        }
+    }
+    for (int n = tid; n < win; n += RS_THREADS) wn[n] = 0.5f - 0.5f * cospif(2.f * (float)n / (float)win);
+    // input stretch of frames t0-3 .. t0+HB-1 in padded coordinates
+    const int c0 = (t0 - 3) * hop;
+    for (int i = tid; i < (NF - 1) * hop + win; i += RS_THREADS) {
+        const int idx = c0 + i - front;
+        xin[i] = (idx >= 0 && idx < N) ? x[idx] : 0.f;
+    }
+    __syncthreads();
+
+    float2 *Z = zbuf + grp * XB, *W = wbuf + grp * XB;
+    const GroupSync gsync{grp + 1, GROUP};
+    for (int pr = grp; 2 * pr < NF; pr += NGROUP) {
+        const int fa = 2 * pr, fb = fa + 1;                       // frame slots; frame number = t0 - 3 + slot
+        const bool have_a = t0 - 3 + fa >= 0 && t0 - 3 + fa < T;
+        const bool have_b = fb < NF && t0 - 3 + fb >= 0 && t0 - 3 + fb < T;
+        if (!have_a && !have_b) continue;                         // (uniform over the group)
+        {
+            float2 v[1][E];
+#pragma unroll
+            for (int r = 0; r < E; ++r) {
+                const int n = tg + GROUP * r;
+                float a = 0.f, b = 0.f;
+                if (n < win) {
+                    const float w = wn[n];
+                    if (have_a) a = w * xin[fa * hop + n];
+                    if (have_b) b = w * xin[fb * hop + n];
+                }
+                v[0][r] = make_float2(a, b);
+            }
+            fft1024_from_regs(v, Z, tg, tw, gsync);
+        }
+        // warped packed spectrum, real and imaginary parts swapped for the inverse
+        for (int k = tg; k <= K / 2; k += GROUP) {
+            const int k0 = k0_s[k];
+            const float fr = fr_s[k], om = 1.f - fr;
+            const float2 z0 = Z[pad0(k0)], z1 = Z[pad0(k0 + 1)];
+            W[pad0(k)] = make_float2(fmaf(fr, z1.y, om * z0.y), fmaf(fr, z1.x, om * z0.x));
+            if (k > 0 && k < K / 2) {
+                const float2 m0 = Z[pad0((K - k0) & (K - 1))], m1 = Z[pad0(K - k0 - 1)];
+                W[pad0(K - k)] = make_float2(fmaf(fr, m1.y, om * m0.y), fmaf(fr, m1.x, om * m0.x));
+            }
+        }
+        gsync();
+        fft1024_in_place(W, tg, tw, gsync);
+        for (int n = tg; n < win; n += GROUP) {
+            const float2 z = W[pad0(n)];                           // (imaginary, real) of the inverse, times K
+            const float w = wn[n] * (1.f / (float)K);
+            if (have_a) fout[fa * win + n] = w * z.y;
+            if (have_b) fout[fb * win + n] = w * z.x;
+        }
+        gsync();      // the buffers are refilled by the group's next pair
+    }
+    __syncthreads();
+
+    // owned samples: hops t0 .. t0+HB-1; sample c is covered by frames c/hop - 3 .. c/hop
+    for (int i = tid; i < HB * hop; i += RS_THREADS) {
+        const int c = t0 * hop + i;
+        const int idx = c - front;
+        if (idx < 0 || idx >= N) continue;
+        const int hb = t0 + i / hop;
+        float acc = 0.f, norm = 0.f;
+#pragma unroll
+        for (int d = 0; d < 4; ++d) {
+            const int t = hb - d;
+            if (t >= 0 && t < T) {
+                const int n = c - t * hop;
+                const float w = wn[n];
+                acc += fout[(t - (t0 - 3)) * win + n];
+                norm = fmaf(w, w, norm);
+            }
+        }
+        y[idx] = acc / norm;
+    }
+}
+
+}  // namespace
+
+int launch_vtlp_resynth(AugCtx *ctx, const float *speech, int64_t stride, const int *lengths,
+                        const AugUttParams *table, int B, int max_len, float *out, int64_t out_stride) {
+    const int win = ctx->cfg.vtlp_win;
+    if (win <= 0 || max_len <= 0) return AUG_OK;
+    const int hop = win / 4, front = win - hop;
+    const int T_cap = (max_len + front + hop - 1) / hop;
+    const size_t smem = resynth_smem(win);
+    if (smem_opt_in<vtlp_resynth_kernel>(ctx->device) != AUG_OK) return AUG_ECUDA;
+    dim3 grid((T_cap + HB - 1) / HB, B);
+    vtlp_resynth_kernel<<<grid, RS_THREADS, smem, ctx->stream>>>(speech, stride, lengths, table, win, ctx->tw,
+                                                                out, out_stride, max_len);
+    AUG_CUDA_OK(cudaGetLastError());
+    ctx->launches++;
+    return AUG_OK;
+}

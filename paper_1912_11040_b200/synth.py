@@ -194,6 +194,29 @@ def sample_table(rng, lengths, bank_len, *, room_lo, room_hi, t60, order,
     return tab
 
 
+def redraw_noise_stretches(table: np.ndarray, lengths: np.ndarray, bank_len: int, seed: int = 0,
+                           min_noise_len: int = 4000, noise_align: int = 1) -> np.ndarray:
+    """A copy of `table` whose noise stretches are drawn again (same ranges as
+    sample_table, own random stream) with offsets and lengths on multiples of
+    `noise_align` samples; everything else is kept.  Used to time and check the same
+    audio with stretches that start and end anywhere."""
+    rng = np.random.default_rng(seed + 7919)
+    tab = table.copy()
+    for b in range(len(tab)):
+        n = int(lengths[b])
+        for j in range(int(tab[b]["n_src"]) - 1):
+            hi = max(min_noise_len, min(n, bank_len))
+            lo = max(min_noise_len, hi // 2)
+            ln = min(int(rng.integers(lo, hi + 1)), bank_len)
+            off = int(rng.integers(0, bank_len - ln + 1))
+            if noise_align > 1:
+                ln = max(noise_align, ln // noise_align * noise_align)
+                off = off // noise_align * noise_align
+            tab[b]["noise_len"][j] = ln
+            tab[b]["noise_offset"][j] = off
+    return tab
+
+
 # --------------------------------------------------------------------------
 # the five named workloads
 # --------------------------------------------------------------------------

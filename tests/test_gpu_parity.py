@@ -293,6 +293,54 @@ def test_pipeline_edge_lengths_and_no_noise():
     assert np.max(np.abs((F - F2).cpu().numpy())) < 1e-3
 
 
+@pytest.mark.parametrize("win", [800, 400])
+def test_waveform_warp_matches_checker(win):
+    """The warp of Eq. 1 applied to the speech waveform with resynthesis: utterances of
+    awkward lengths (one sample, just under / at / over a hop and a window, several CTAs'
+    worth), warp factors on both sides of 1 and 1 itself (which must return the input)."""
+    import torch
+    w = small(2, batch=8, dur_scale=0.12)
+    w.cfg["vtlp_win"] = win
+    hop = win // 4
+    w.lengths[:6] = [1, hop - 1, hop, win + 1, 3 * win + 7, 0]
+    w.table["alpha"][:8] = [0.8, 1.2, 0.93, 1.07, 1.0, 0.9, 0.85, 1.15]
+    dev = Device(w)
+    out = torch.full_like(dev.speech, float("nan"))
+    dev.ctx.aug_vtlp_resynth(dev.speech, w.stride, dev.lengths, dev.table, w.B, out, w.stride)
+    torch.cuda.synchronize()
+    out = out.cpu().numpy()
+    for b in range(w.B):
+        n = int(w.lengths[b])
+        ref = oracle.vtlp_resynth(w.speech[b, :n].astype(np.float64), float(w.table[b]["alpha"]), win)
+        check_wave(out[b, :n], ref, f"utt {b}")
+        assert np.all(np.isnan(out[b, n:]))
+    b = 4                                               # alpha = 1: the input comes back
+    n = int(w.lengths[b])
+    assert np.max(np.abs(out[b, :n] - w.speech[b, :n])) <= 1e-5 * np.sqrt(np.mean(w.speech[b, :n] ** 2))
+    # a context without the option refuses the call
+    w2 = small(1, batch=1, dur_scale=0.1)
+    dev2 = Device(w2)
+    o2 = torch.zeros_like(dev2.speech)
+    assert dev2.ctx.aug_vtlp_resynth(dev2.speech, w2.stride, dev2.lengths, dev2.table, 1, o2, w2.stride,
+                                     check=False) == binding.AUG_EINVAL
+
+
+def test_pipeline_with_the_waveform_warp():
+    """vtlp_win > 0: speech is warped before the simulator (noise and reverberation are
+    not), the filterbank stays unwarped; whole path against the checker."""
+    w = small(2, **REDUCED[2])
+    w.cfg["vtlp_win"] = 800
+    dev = Device(w)
+    F, counts, wave = dev.pipeline(want_wave=True)
+    assert dev.ctx.aug_last_status() == (-1, 0)
+    worst_f, worst_w = check_pipeline_against_oracle(dev, F, counts, wave, oracle_batch(w))
+    print(f"waveform warp: worst log-mel err {worst_f:.2e}, worst wave err/rms {worst_w:.2e}")
+    # and it differs from warping inside the filterbank
+    w0 = small(2, **REDUCED[2])
+    F0, _, _ = Device(w0).pipeline(want_wave=False)
+    assert float((F - F0).abs().max()) > 0.05
+
+
 def test_power_law_compression():
     w = small(1, batch=2)
     dev = Device(w, compression=binding.COMPRESS_POW_1_15)
