@@ -131,8 +131,8 @@ int aug_validate_params(const AugConfig *cfg_host, const AugUttParams *table_hos
                         int64_t bank_len, int *bad_row_host);
 
 /* Ranges the per-utterance parameters are drawn from (uniformly, independently):
- * the "millions of room dimensions, wide distribution of reverberation time and
- * SNR" of Section 1 and the random warp factor of Section 2.3. */
+ * the variety of room sizes, reverberation times and SNRs that Section 1 describes
+ * for the simulator, and the random warp factor of Section 2.3. */
 typedef struct {
     float room_lo[3], room_hi[3]; /* shoebox side lengths, metres */
     float t60_lo, t60_hi;         /* reverberation time, seconds; turned into one wall reflection

@@ -102,8 +102,8 @@ Layout make_layout(const AugConfig &c) {
     l.off_xspec = l.route == aug::ROUTE_STORED ? take(sizeof(float2) * B * S * l.nblk_cap * aug::CONV_N2) : -1;
     // parking slots of the fused route, three per multiprocessor, when a row can have several noises
     const bool parks = l.route == aug::ROUTE_FUSED_8192 && c.max_sources >= 3;
-    l.off_park = parks ? take(sizeof(float2) * (int64_t)aug::PARK_SMS * 3 * 2 * aug::CONV_N2) : -1;
-    l.off_park_flags = parks ? take(sizeof(int) * (int64_t)aug::PARK_SMS * 3) : -1;
+    l.off_park = parks ? take(sizeof(float2) * (int64_t)aug::PARK_SMS * aug::PARK_PER_SM * 2 * aug::CONV_N2) : -1;
+    l.off_park_flags = parks ? take(sizeof(int) * (int64_t)aug::PARK_SMS * aug::PARK_PER_SM) : -1;
     l.off_ys = take(sizeof(float) * B * l.ws_stride);
     l.off_vv = take(sizeof(float) * B * l.ws_stride);
     l.off_energy = take(sizeof(double) * 2 * B);
@@ -276,7 +276,8 @@ int aug_create(AugCtx **out, const AugConfig *cfg, void *cuda_stream) {
     }
     const int st0[2] = {-1, 0};
     if (ctx->park_flags &&
-        cudaMemsetAsync(ctx->park_flags, 0, sizeof(int) * aug::PARK_SMS * 3, ctx->stream) != cudaSuccess) {
+        cudaMemsetAsync(ctx->park_flags, 0, sizeof(int) * aug::PARK_SMS * aug::PARK_PER_SM, ctx->stream) !=
+            cudaSuccess) {
         cudaFree(ctx->ws_base);
         delete ctx;
         return AUG_ECUDA;
@@ -464,7 +465,7 @@ int aug_pipeline(AugCtx *ctx, const float *speech_dev, int64_t speech_stride,
         return rc;
     t1(5, sm);
     t0(6, sm);
-    rc = launch_fused_features(ctx, lengths_dev, table_dev, B, feats_dev, T_max, frame_counts_dev);
+    rc = launch_fused_features(ctx, lengths_dev, table_dev, B, feats_dev, T_max, frame_counts_dev, max_len);
     t1(6, sm);
     if (ev && rc == AUG_OK) ctx->ev_n++;
     return rc;
@@ -588,7 +589,7 @@ int aug_hold_parking_slots(AugCtx *ctx, int hold) {
     if (!ctx) return AUG_EINVAL;
     if (!ctx->park_flags) return AUG_OK;   // this context has no parking area
     // all slots marked taken: every CTA then sums its noise sources in the time domain
-    std::vector<int> v((size_t)aug::PARK_SMS * 3, hold ? 1 : 0);
+    std::vector<int> v((size_t)aug::PARK_SMS * aug::PARK_PER_SM, hold ? 1 : 0);
     AUG_CUDA_OK(cudaStreamSynchronize(ctx->stream));
     AUG_CUDA_OK(cudaMemcpyAsync(ctx->park_flags, v.data(), sizeof(int) * v.size(), cudaMemcpyHostToDevice,
                                 ctx->stream));

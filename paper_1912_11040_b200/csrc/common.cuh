@@ -12,7 +12,8 @@ namespace aug {
 constexpr int CONV_BLK = 4096;          // output samples per convolution block
 constexpr int CONV_F = 2 * CONV_BLK;    // real FFT size of one block
 constexpr int CONV_N2 = CONV_F / 2;     // complex FFT size
-constexpr int PARK_SMS = 160;       // multiprocessors that get parking slots (3 each) in the fused convolution
+constexpr int PARK_SMS = 160;       // multiprocessors that get parking slots in the fused convolution
+constexpr int PARK_PER_SM = 3;      // slots per multiprocessor = resident CTAs of that kernel
 constexpr int MAX_TAPS = 24576;
 constexpr int MAX_ORDER = 32;
 constexpr int MAX_HALF_W = 47;
@@ -60,8 +61,8 @@ struct AugCtx {
     float2 *hspec;         // [max_batch][max_sources][n_part][CONV_N2]
     float2 *xspec;         // [max_batch][max_sources][nblk_cap][CONV_N2]; NULL unless route == ROUTE_STORED
     int nblk_cap;          // blocks of an utterance of max_samples
-    float2 *park;          // [PARK_SMS * 3][8192] products of noise sources waiting for the last one; NULL if unused
-    int *park_flags;       // [PARK_SMS * 3] 1 = slot taken
+    float2 *park;          // [PARK_SMS * PARK_PER_SM][8192] products of noise sources waiting for the last one; NULL if unused
+    int *park_flags;       // [PARK_SMS * PARK_PER_SM] 1 = slot taken
     int n_sm;              // multiprocessors with slots (PARK_SMS); CTAs on others sum in the time domain
     float *warped;         // [max_batch][ws_stride] speech after the waveform warp; NULL unless cfg.vtlp_win
     float *ys;             // [max_batch][ws_stride]
@@ -138,4 +139,4 @@ int launch_stft_power(AugCtx *ctx, const float *wave, int64_t stride, const int 
 int launch_logmel(AugCtx *ctx, const float *power, const int *counts, int B, int T_max,
                   float *feats);
 int launch_fused_features(AugCtx *ctx, const int *lengths, const AugUttParams *table, int B,
-                          float *feats, int T_max, int *counts);
+                          float *feats, int T_max, int *counts, int max_len);

@@ -41,6 +41,7 @@ constexpr int SM_POINTS = padded_points(N2);
 #ifndef CONV_MINB
 #define CONV_MINB 3                  // CTAs per SM the register budget is set for
 #endif
+static_assert(CONV_MINB == aug::PARK_PER_SM, "one parking slot per resident CTA of the fused convolution");
 
 __device__ __forceinline__ void fft4096_from_regs(float2 (*v)[E], float2 *s, int t,
                                                   const float2 *__restrict__ tw) {

@@ -695,7 +695,7 @@ logmel_kernel(const float *__restrict__ power, const int *__restrict__ counts, i
 
 template <int K, int MODE>
 int launch_frames(AugCtx *ctx, const float *a, const float *b, int64_t stride, const int *lengths,
-                  const AugUttParams *table, int B, float *out, int T_max, int *counts) {
+                  const AugUttParams *table, int B, float *out, int T_max, int *counts, int n_cap) {
     const AugConfig &c = ctx->cfg;
     constexpr int FT = Plan<K>::FT, NBP = K / 2 + 1;
     const int chunk_cap = ((FT - 1) * c.hop + c.win + 3) & ~3;
@@ -717,7 +717,7 @@ int launch_frames(AugCtx *ctx, const float *a, const float *b, int64_t stride, c
     kern<<<grid, FEAT_THREADS, smem, ctx->stream>>>(
         a, b, stride, ctx->gain, table, lengths, c.win, c.hop, c.n_mel, T_max, ctx->melw,
         ctx->melstart, ctx->tw, c.log_floor, c.pad_value, c.compression, out, counts,
-        (int)(stride < 0x7fffffff ? stride : 0x7fffffff));
+        n_cap);
     AUG_CUDA_OK(cudaGetLastError());
     ctx->launches++;
     return AUG_OK;
@@ -738,9 +738,10 @@ int launch_mel_tables(AugCtx *ctx, const AugUttParams *table, int B, cudaStream_
 int launch_stft_power(AugCtx *ctx, const float *wave, int64_t stride, const int *lengths, int B,
                       float *power, int T_max, int *counts) {
     if (T_max <= 0) return AUG_OK;
+    const int n_cap = (int)(stride < 0x7fffffff ? stride : 0x7fffffff);     // the caller's rows end at their stride
     if (ctx->cfg.n_fft == 512)
-        return launch_frames<512, 0>(ctx, wave, nullptr, stride, lengths, nullptr, B, power, T_max, counts);
-    return launch_frames<1024, 0>(ctx, wave, nullptr, stride, lengths, nullptr, B, power, T_max, counts);
+        return launch_frames<512, 0>(ctx, wave, nullptr, stride, lengths, nullptr, B, power, T_max, counts, n_cap);
+    return launch_frames<1024, 0>(ctx, wave, nullptr, stride, lengths, nullptr, B, power, T_max, counts, n_cap);
 }
 
 #ifndef FEAT_WP_TILES
@@ -748,7 +749,8 @@ int launch_stft_power(AugCtx *ctx, const float *wave, int64_t stride, const int 
 #endif
 
 // Fused features with the 512-point transform: the warp-per-frame-pair kernel.
-static int launch_frames_warp(AugCtx *ctx, const int *lengths, int B, float *feats, int T_max, int *counts) {
+static int launch_frames_warp(AugCtx *ctx, const int *lengths, int B, float *feats, int T_max, int *counts,
+                              int max_len) {
     const AugConfig &c = ctx->cfg;
     const size_t smem = wp::smem_bytes(c.win, c.hop, c.n_mel);
     if (smem > 227 * 1024) return AUG_ECAP;
@@ -762,24 +764,25 @@ static int launch_frames_warp(AugCtx *ctx, const int *lengths, int B, float *fea
         return AUG_ECUDA;
     kern<<<grid, FEAT_THREADS, smem, ctx->stream>>>(
         ctx->ys, ctx->vv, ctx->ws_stride, ctx->gain, lengths, c.win, c.hop, c.n_mel, T_max, ctx->melw,
-        ctx->melstart, ctx->tw, c.log_floor, c.pad_value, c.compression, feats, counts,
-        (int)(ctx->ws_stride < 0x7fffffff ? ctx->ws_stride : 0x7fffffff));
+        ctx->melstart, ctx->tw, c.log_floor, c.pad_value, c.compression, feats, counts, max_len);
     AUG_CUDA_OK(cudaGetLastError());
     ctx->launches++;
     return AUG_OK;
 }
 
+// max_len: the length clamp the convolution used, so that every stage cuts an over-long
+// entry of `lengths` at the same sample.
 int launch_fused_features(AugCtx *ctx, const int *lengths, const AugUttParams *table, int B,
-                          float *feats, int T_max, int *counts) {
+                          float *feats, int T_max, int *counts, int max_len) {
     if (T_max <= 0) return AUG_OK;
 #ifndef FEAT_OLD_512
-    if (ctx->cfg.n_fft == 512) return launch_frames_warp(ctx, lengths, B, feats, T_max, counts);
+    if (ctx->cfg.n_fft == 512) return launch_frames_warp(ctx, lengths, B, feats, T_max, counts, max_len);
 #endif
     if (ctx->cfg.n_fft == 512)
         return launch_frames<512, 1>(ctx, ctx->ys, ctx->vv, ctx->ws_stride, lengths, table, B, feats,
-                                     T_max, counts);
+                                     T_max, counts, max_len);
     return launch_frames<1024, 1>(ctx, ctx->ys, ctx->vv, ctx->ws_stride, lengths, table, B, feats,
-                                  T_max, counts);
+                                  T_max, counts, max_len);
 }
 
 int launch_logmel(AugCtx *ctx, const float *power, const int *counts, int B, int T_max,

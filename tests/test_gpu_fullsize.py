@@ -50,3 +50,20 @@ def test_full_size_workload(index, n_check, noise_align):
     _, worst_w = check_pipeline_against_oracle(dev, F2, counts2, wave, orc)
     print(f"config{index} full size ({w.B} utts, {w.audio_seconds:.0f} audio-s): utterances {picks}: "
           f"worst log-mel err {worst_f:.2e}, worst wave err/rms {worst_w:.2e}")
+
+
+def test_parked_and_time_domain_noise_sums_agree_on_every_utterance():
+    """Config 2 at full size with parking slots under contention (every multiprocessor's
+    slots in use at once): the frequency-domain sum of several noise sources must give
+    the same features, for every utterance of the batch, as the time-domain sum that a CTA
+    falls back to when it finds no slot."""
+    w = synth.make_workload(2, seed=0)
+    dev = Device(w)
+    F1, c1, _ = dev.pipeline(want_wave=False, lengths_host=True)
+    dev.ctx.aug_hold_parking_slots(True)
+    F2, c2, _ = dev.pipeline(want_wave=False, lengths_host=True)
+    dev.ctx.aug_hold_parking_slots(False)
+    assert dev.ctx.aug_last_status() == (-1, 0)
+    assert np.array_equal(c1.cpu().numpy(), c2.cpu().numpy())
+    assert int((w.table["n_src"] > 2).sum()) > 20                 # rows that do use the slots
+    assert float((F1 - F2).abs().max()) <= 1e-3
