@@ -32,15 +32,26 @@ METRIC = "audio-seconds augmented+featurised per second"
 UNIT = "audio-s/s"
 FP32_LANES = 128          # fp32 lanes of one multiprocessor
 
-# DRAM bytes per audio-second of workload 2 (dram__bytes_read.sum + dram__bytes_write.sum of one
-# ncu --set full capture on 96 utterances; traffic grows in proportion to the audio processed).
-# Valid only for the kernel sources the capture was taken from: the hash guards that.
+# DRAM bytes per audio-second (dram__bytes_read.sum + dram__bytes_write.sum of one ncu --set full
+# capture per kernel on a reduced batch: profiles/ncu_config{2,3,5}_kernels.md; traffic grows in
+# proportion to the audio processed).  Valid only for the kernel sources the captures were taken
+# from: the hashes guard that.
 NCU_TRAFFIC = {
-    "workload": 2,
-    "bytes_per_audio_s": {"convolve": 275.28e6 / 1039.18, "features": 152.86e6 / 1039.18},
+    "bytes_per_audio_s": {
+        2: {"convolve": 276.1e6 / 1039.18, "features": 151.3e6 / 1039.18, "rir_image": 45.6e6 / 1039.18},
+        3: {"convolve": 86.7e6 / 128.0, "block_spectra": 30.3e6 / 128.0, "rir_image": 32.8e6 / 128.0},
+        5: {"convolve": 107.9e6 / 240.0, "block_spectra": 75.5e6 / 240.0, "features": 30.8e6 / 240.0}},
+    "captured_on": {2: "96 utterances", 3: "16 utterances", 5: "4 utterances"},
     # kernel -> (its source files, sha256[:16] of them when the counters were taken)
-    "sources": {"convolve": (("conv.cu", "fft.cuh"), "1d0dd1be6958f74a"),
-                "features": (("feat.cu", "fft.cuh"), "a0a6419dbd470497")}}
+    "sources": {"convolve": (("conv.cu", "fft.cuh"), "a614026f276abea4"),
+                "block_spectra": (("conv.cu", "fft.cuh"), "a614026f276abea4"),
+                "features": (("feat.cu", "fft.cuh"), "995cd357c5095026"),
+                "rir_image": (("rir.cu",), "e530344d7f3587b9")}}
+
+
+# nominal FMAs / fp32 instructions executed: convolution 480 / 736 per thread and 4096-point
+# transform; fused 512-point features 6274 / 11680 per frame
+FP32_INSTRUCTION_CEILING = {"convolve": 0.652, "block_spectra": 0.652, "features": 0.537}
 
 
 def kernel_sources_sha(files):
@@ -521,6 +532,12 @@ def run_ours(args):
             "ms": ms, "bound": bound,
             "tflops": flops / (ms * 1e-3) / 1e12, "frac_fp32": flops / (ms * 1e-3) / 1e12 / fp32_measured,
             "gbs": byts / (ms * 1e-3) / 1e9, "frac_hbm": byts / (ms * 1e-3) / 1e9 / hbm_peak}
+    # fp32 instructions executed per nominal FMA (ncu instruction counts in profiles/): no SIMT
+    # kernel that issues one instruction per slot can exceed this share of the nominal-flop roofline
+    for name, ceil in FP32_INSTRUCTION_CEILING.items():
+        if name in per_kernel and not (name == "features" and int(w.cfg["n_fft"]) != 512):
+            per_kernel[name]["fp32_instruction_ceiling"] = ceil
+            per_kernel[name]["frac_of_instruction_ceiling"] = per_kernel[name]["frac_fp32"] / ceil
     d = per_kernel[dom]
     if d["bound"] == "alu":
         roofline = {"kernel": dom, "bound": "alu", "achieved": d["tflops"], "peak": fp32_measured,
@@ -531,11 +548,13 @@ def run_ours(args):
         roofline = {"kernel": dom, "bound": "hbm", "achieved": d["gbs"], "peak": hbm_peak,
                     "unit": "GB/s", "frac": d["frac_hbm"], "traffic": None,
                     "peak_source": f"{hbm_src} copy bandwidth"}
-    if (args.workload == NCU_TRAFFIC["workload"] and dom in NCU_TRAFFIC["bytes_per_audio_s"]
+    per_audio = NCU_TRAFFIC["bytes_per_audio_s"].get(args.workload, {})
+    if (dom in per_audio and args.vtlp_win == 0
             and kernel_sources_sha(NCU_TRAFFIC["sources"][dom][0]) == NCU_TRAFFIC["sources"][dom][1]):
-        roofline["traffic"] = NCU_TRAFFIC["bytes_per_audio_s"][dom] * w.audio_seconds
-        roofline["traffic_note"] = ("bytes per launch, ncu capture on 96 utterances scaled by audio-seconds; "
-                                    "algorithmic bytes of this kernel: %.3e" % kernels[dom][1][1])
+        roofline["traffic"] = per_audio[dom] * w.audio_seconds
+        roofline["traffic_note"] = ("bytes per launch, ncu capture on %s scaled by audio-seconds; "
+                                    "algorithmic bytes of this kernel: %.3e"
+                                    % (NCU_TRAFFIC["captured_on"][args.workload], kernels[dom][1][1]))
     roofline["per_kernel"] = per_kernel
     roofline["stage_ms"] = dict(zip(binding.STAGE_NAMES, stage_ms))
     roofline["stage_calls_averaged"] = n_rec
