@@ -80,7 +80,7 @@ struct Layout {
     int n_part, route, n_bins, t_cap, nblk_cap;
     int64_t ws_stride;
     int64_t off_xspec, off_park, off_park_flags;
-    int64_t off_tw, off_rir, off_hspec, off_ys, off_vv, off_energy, off_gain, off_melw, off_melstart,
+    int64_t off_tw, off_rir, off_hspec, off_ys, off_vv, off_energy, off_leff, off_gain, off_melw, off_melstart,
         off_status, off_warped, off_st_speech, off_st_bank, off_st_table, off_st_lengths,
         off_st_feats, off_st_counts, total;
 };
@@ -107,6 +107,7 @@ Layout make_layout(const AugConfig &c) {
     l.off_ys = take(sizeof(float) * B * l.ws_stride);
     l.off_vv = take(sizeof(float) * B * l.ws_stride);
     l.off_energy = take(sizeof(double) * 2 * B);
+    l.off_leff = take(sizeof(int) * B);
     l.off_gain = take(sizeof(float) * B);
     l.off_melw = take(sizeof(aug::MelBin) * B * l.n_bins);
     l.off_melstart = take(sizeof(int) * B * (c.n_mel + 2));
@@ -239,6 +240,7 @@ int aug_create(AugCtx **out, const AugConfig *cfg, void *cuda_stream) {
     ctx->ys = reinterpret_cast<float *>(base + l.off_ys);
     ctx->vv = reinterpret_cast<float *>(base + l.off_vv);
     ctx->energy = reinterpret_cast<double *>(base + l.off_energy);
+    ctx->leff = reinterpret_cast<int *>(base + l.off_leff);
     ctx->gain = reinterpret_cast<float *>(base + l.off_gain);
     ctx->melw = reinterpret_cast<aug::MelBin *>(base + l.off_melw);
     ctx->melstart = reinterpret_cast<int *>(base + l.off_melstart);

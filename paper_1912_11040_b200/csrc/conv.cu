@@ -21,6 +21,13 @@
 //                     and inverse-transforms.  Noise sources are summed in the
 //                     frequency domain: two inverse transforms per block.
 //
+// Responses are often shorter than their buffer: behind the last image source's window
+// every tap is exactly zero.  The kernels that transform the responses record, per
+// utterance, the number of taps up to the last non-zero one (the largest over its
+// sources); the fused route then takes 16384 - that + 1 outputs from every block
+// instead of 16384 - rir_taps + 1, and the stored-spectra route skips the partitions
+// that are zero throughout.  The result is the same convolution.
+//
 // A real transform of F points is a complex transform of F/2 points on (even, odd)
 // sample pairs followed by the usual split; in the 8192-point routes thread t owns
 // the bin pairs (k, F/2-k), k = t + 256 q.  Spectra are stored as F/2 complex numbers
@@ -220,11 +227,26 @@ __device__ __forceinline__ void finish_block(const float2 (*acc)[2], float2 *sm,
     __syncthreads();
 }
 
+// Largest (index + 1) of a non-zero tap seen by the CTA -> leff[utt] (atomic maximum).
+__device__ __forceinline__ void record_length(int last_plus_1, int *leff_slot, int *red_i, int t) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) last_plus_1 = max(last_plus_1, __shfl_xor_sync(0xffffffffu, last_plus_1, o));
+    if ((t & 31) == 0) red_i[t >> 5] = last_plus_1;
+    __syncthreads();
+    if (t == 0) {
+        int m = 0;
+        for (int i = 0; i < CT / 32; ++i) m = max(m, red_i[i]);
+        if (m > 0) atomicMax(leff_slot, m);
+    }
+}
+
 // ---------------------------------------------------------------- partition spectra
 __global__ void __launch_bounds__(CT)
 rir_spectra_kernel(const float *__restrict__ rir, const AugUttParams *__restrict__ table, int S_max,
-                   int L, int P, const float2 *__restrict__ tw, float2 *__restrict__ hspec) {
+                   int L, int P, const float2 *__restrict__ tw, float2 *__restrict__ hspec,
+                   int *__restrict__ leff) {
     extern __shared__ __align__(16) float2 sm[];
+    __shared__ int red_i[CT / 32];
     const int p = blockIdx.x, s = blockIdx.y, utt = blockIdx.z, t = threadIdx.x;
     const AugUttParams &row = table[utt];
     if (row.n_src < 1 || row.n_src > S_max || s >= row.n_src) return;
@@ -233,6 +255,7 @@ rir_spectra_kernel(const float *__restrict__ rir, const AugUttParams *__restrict
     float2 *out = hspec + (((int64_t)utt * S_max + s) * P + p) * N2;
 
     float2 v[1][E];
+    int last = 0;
 #pragma unroll
     for (int r = 0; r < E; ++r) {
         const int n = t + CT * r;                 // complex index; taps 2n, 2n+1 of the partition
@@ -241,9 +264,12 @@ rir_spectra_kernel(const float *__restrict__ rir, const AugUttParams *__restrict
         if (n < BLK / 2) {
             if (i0 < L) z.x = h[i0];
             if (i0 + 1 < L) z.y = h[i0 + 1];
+            if (z.x != 0.f) last = max(last, i0 + 1);
+            if (z.y != 0.f) last = max(last, i0 + 2);
         }
         v[0][r] = z;
     }
+    record_length(last, &leff[utt], red_i, t);
     fft4096_from_regs(v, sm, t, tw);
 #pragma unroll
     for (int q = 0; q < NQ; ++q) {
@@ -295,10 +321,12 @@ spectral_convolve_kernel(const int *__restrict__ lengths, const float *__restric
                          const float2 *__restrict__ hspec, const float2 *__restrict__ xspec,
                          int nblk_cap, const float2 *__restrict__ tw, float *__restrict__ ys,
                          float *__restrict__ vv, int64_t ws_stride, double *__restrict__ energy,
-                         int n_cap) {
+                         int n_cap, const int *__restrict__ leff) {
     extern __shared__ __align__(16) float2 sm[];
     __shared__ float red[CT / 32];
     const int b = blockIdx.x, utt = blockIdx.y, t = threadIdx.x;
+    // partitions behind the last non-zero tap of every source of this utterance are zero
+    const int P_used = min(P, (max(leff[utt], 1) + BLK - 1) / BLK);
     const int N = min(max(lengths[utt], 0), n_cap);
     if ((int64_t)b * BLK >= N) return;
     const AugUttParams &row = table[utt];
@@ -317,7 +345,7 @@ spectral_convolve_kernel(const int *__restrict__ lengths, const float *__restric
             if (!source_of(row, s, nullptr, bank, bank_len, x, nlen)) continue;   // no spectra stored
             const float2 *Hs = hspec + ((int64_t)utt * S_max + s) * P * N2;
             const float2 *Xs = xspec + ((int64_t)utt * S_max + s) * nblk_cap * N2;
-            for (int p = 0; p < P && p <= b; ++p) {
+            for (int p = 0; p < P_used && p <= b; ++p) {
                 const float2 *H = Hs + (int64_t)p * N2;
                 const float2 *X = Xs + (int64_t)(b - p) * N2;
 #pragma unroll
@@ -598,8 +626,10 @@ __device__ __forceinline__ void edge_inverse(const Edge &y, float2 uh, float2 &a
 // the whole second half are zero), scaled by the noise weight and 1/F.
 __global__ void __launch_bounds__(CT)
 rir_spectra2_kernel(const float *__restrict__ rir, const AugUttParams *__restrict__ table, int S_max,
-                    int L, const float2 *__restrict__ tw, float2 *__restrict__ hspec) {
+                    int L, const float2 *__restrict__ tw, float2 *__restrict__ hspec,
+                    int *__restrict__ leff) {
     extern __shared__ __align__(16) float2 sm[];
+    __shared__ int red_i[CT / 32];
     float2 *A = sm, *Bf = sm + SM_POINTS;
     const int s = blockIdx.x, utt = blockIdx.y, t = threadIdx.x;
     const AugUttParams &row = table[utt];
@@ -609,6 +639,7 @@ rir_spectra2_kernel(const float *__restrict__ rir, const AugUttParams *__restric
     float2 *out = hspec + ((int64_t)utt * S_max + s) * NB2;
     {
         float2 va[1][E], vb[1][E];
+        int last = 0;
 #pragma unroll
         for (int r = 0; r < E; ++r) {
             const int i0 = 4 * (t + CT * r);
@@ -618,10 +649,15 @@ rir_spectra2_kernel(const float *__restrict__ rir, const AugUttParams *__restric
                 if (i0 + 1 < L) z.y = h[i0 + 1];
                 if (i0 + 2 < L) z.z = h[i0 + 2];
                 if (i0 + 3 < L) z.w = h[i0 + 3];
+                if (z.x != 0.f) last = max(last, i0 + 1);
+                if (z.y != 0.f) last = max(last, i0 + 2);
+                if (z.z != 0.f) last = max(last, i0 + 3);
+                if (z.w != 0.f) last = max(last, i0 + 4);
             }
             va[0][r] = make_float2(z.x, z.y);
             vb[0][r] = make_float2(z.z, z.w);
         }
+        record_length(last, &leff[utt], red_i, t);
         fft2x4096_from_regs(va, vb, A, Bf, t, tw);
         __syncthreads();
     }
@@ -674,14 +710,17 @@ convolve_fused2_kernel(const float *__restrict__ speech, int64_t stride,
                        int64_t bank_len, const AugUttParams *__restrict__ table, int S_max,
                        const float2 *__restrict__ hspec, const float2 *__restrict__ tw,
                        float *__restrict__ ys, float *__restrict__ vv, int64_t ws_stride,
-                       double *__restrict__ energy, int *status, int n_cap, int ob,
-                       float2 *__restrict__ park, int *park_flags, int n_sm) {
+                       double *__restrict__ energy, int *status, int n_cap,
+                       const int *__restrict__ leff, float2 *__restrict__ park, int *park_flags, int n_sm) {
     extern __shared__ __align__(16) float2 sm[];
     float2 *A = sm, *Bf = sm + SM_POINTS;
     __shared__ float red[CT / 32];
     __shared__ int park_slot_s;
     const int b = blockIdx.x, utt = blockIdx.y, t = threadIdx.x;
     const int N = min(max(lengths[utt], 0), n_cap);
+    // every block yields the F2 - (taps - 1) outputs that see no wrap-around, cut to a multiple
+    // of 4, where taps counts up to the last non-zero tap of this utterance's responses
+    const int ob = (F2 - min(max(leff[utt], 1), BLK2) + 1) & ~3;
     if ((int64_t)b * ob >= N) return;
     const AugUttParams &row = table[utt];
     int n_src = row.n_src;
@@ -861,15 +900,16 @@ constexpr size_t FFT2_SMEM = 2 * FFT_SMEM;
 int launch_rir_spectra(AugCtx *ctx, const float *rir, const AugUttParams *table, int B,
                        cudaStream_t st) {
     const AugConfig &c = ctx->cfg;
+    AUG_CUDA_OK(cudaMemsetAsync(ctx->leff, 0, sizeof(int) * (size_t)B, st));
     if (ctx->route == aug::ROUTE_FUSED_8192) {
         if (smem_opt_in<rir_spectra2_kernel>(ctx->device) != AUG_OK) return AUG_ECUDA;
         dim3 grid(c.max_sources, B);
         rir_spectra2_kernel<<<grid, CT, FFT2_SMEM, st>>>(rir, table, c.max_sources, c.rir_taps, ctx->tw,
-                                                         ctx->hspec);
+                                                         ctx->hspec, ctx->leff);
     } else {
         dim3 grid(ctx->n_part, c.max_sources, B);
         rir_spectra_kernel<<<grid, CT, FFT_SMEM, st>>>(rir, table, c.max_sources, c.rir_taps,
-                                                       ctx->n_part, ctx->tw, ctx->hspec);
+                                                       ctx->n_part, ctx->tw, ctx->hspec, ctx->leff);
     }
     AUG_CUDA_OK(cudaGetLastError());
     ctx->launches++;
@@ -903,9 +943,9 @@ int launch_convolve_finish(AugCtx *ctx, const float *speech, int64_t stride, con
     const int nblk = (max_len + BLK - 1) / BLK;
     dim3 grid(nblk, B);
     if (ctx->route == aug::ROUTE_FUSED_8192) {
-        // every block yields the F2 - (taps - 1) outputs that see no wrap-around, cut to a multiple of 4
-        const int ob = (F2 - c.rir_taps + 1) & ~3;
-        const int nblk2 = (max_len + ob - 1) / ob;
+        // the grid covers the shortest block any utterance can have (a response that fills its buffer)
+        const int ob_min = (F2 - c.rir_taps + 1) & ~3;
+        const int nblk2 = (max_len + ob_min - 1) / ob_min;
         dim3 grid2(nblk2, B);
         auto kern = ctx->park ? convolve_fused2_kernel<true> : convolve_fused2_kernel<false>;
         if ((ctx->park ? smem_opt_in<convolve_fused2_kernel<true>>(ctx->device)
@@ -913,12 +953,12 @@ int launch_convolve_finish(AugCtx *ctx, const float *speech, int64_t stride, con
             return AUG_ECUDA;
         kern<<<grid2, CT, FFT2_SMEM, ctx->stream>>>(
             speech, stride, lengths, bank, bank_len, table, c.max_sources, ctx->hspec, ctx->tw,
-            ctx->ys, ctx->vv, ctx->ws_stride, ctx->energy, ctx->status, max_len, ob, ctx->park,
+            ctx->ys, ctx->vv, ctx->ws_stride, ctx->energy, ctx->status, max_len, ctx->leff, ctx->park,
             ctx->park_flags, ctx->n_sm);
     } else {
         spectral_convolve_kernel<<<grid, CT, FFT_SMEM, ctx->stream>>>(
             lengths, bank, bank_len, table, c.max_sources, ctx->n_part, ctx->hspec, ctx->xspec,
-            ctx->nblk_cap, ctx->tw, ctx->ys, ctx->vv, ctx->ws_stride, ctx->energy, max_len);
+            ctx->nblk_cap, ctx->tw, ctx->ys, ctx->vv, ctx->ws_stride, ctx->energy, max_len, ctx->leff);
     }
     AUG_CUDA_OK(cudaGetLastError());
     ctx->launches++;
