@@ -173,6 +173,36 @@ def test_reverb_mix_matches_direct_convolution(index):
         assert np.all(np.isnan(out[b, n:]))          # samples beyond the length are untouched
 
 
+@pytest.mark.parametrize("index", [2, 5])
+def test_reverb_mix_with_responses_of_any_effective_length(index):
+    """The convolution sizes its blocks (fused route) or skips partitions (stored-spectra
+    route) by the last non-zero tap of an utterance's responses.  Caller-supplied responses
+    that are a single tap at 0, a single tap at the very end of the buffer, dense to the
+    last tap, and all zero must all give the plain convolution."""
+    import torch
+    w = small(index, **dict(REDUCED[index], batch=5))
+    w.table["n_src"][:] = 2
+    dev = Device(w)
+    L = dev.L
+    rng = np.random.default_rng(11)
+    rir = np.zeros((w.B, dev.S, L), dtype=np.float32)
+    rir[0, 0, 0], rir[0, 1, 0] = 0.7, -0.4                       # one tap at 0: effective length 1
+    rir[1, 0, L - 1], rir[1, 1, 3] = 0.5, 0.25                   # last tap of the buffer
+    rir[2, :2] = rng.standard_normal((2, L)) * np.exp(-np.arange(L) / (0.2 * L)) * 0.05   # dense to the end
+    rir[3, 0, : L // 3] = rng.standard_normal(L // 3) * 0.05     # speech response short, noise response long
+    rir[3, 1, : L - 7] = rng.standard_normal(L - 7) * 0.05
+    # utterance 4: all-zero responses
+    out = dev.reverb_mix(torch.from_numpy(rir).cuda()).cpu().numpy()
+    for b in range(w.B):
+        n = int(w.lengths[b])
+        noise = oracle.looped_noise(w.bank, w.table[b]["noise_offset"][0], w.table[b]["noise_len"][0], n)
+        ref, *_ = oracle.reverb_mix(w.speech[b, :n].astype(np.float64),
+                                    [rir[b, 0].astype(np.float64), rir[b, 1].astype(np.float64)], [noise],
+                                    w.table[b]["noise_weight"], w.table[b]["snr_db"])
+        check_wave(out[b, :n], ref, f"cfg{index} utt {b}")
+    assert not out[4, : int(w.lengths[4])].any()
+
+
 @pytest.mark.parametrize("index", [1, 5])
 def test_stft_power_and_logmel_match(index):
     w = small(index, **REDUCED[index]) if index != 1 else small(1, batch=4)
