@@ -101,13 +101,13 @@ Layout make_layout(const AugConfig &c) {
     l.nblk_cap = (c.max_samples + aug::CONV_BLK - 1) / aug::CONV_BLK;
     l.off_xspec = l.route == aug::ROUTE_STORED ? take(sizeof(float2) * B * S * l.nblk_cap * aug::CONV_N2) : -1;
     // parking slots of the fused route, three per multiprocessor, when a row can have several noises
-    const bool parks = l.route == aug::ROUTE_FUSED_8192 && c.max_sources >= 3;
+    const bool parks = c.max_sources >= 3;    // (long-response contexts use the fused route for short responses)
     l.off_park = parks ? take(sizeof(float2) * (int64_t)aug::PARK_SMS * aug::PARK_PER_SM * 2 * aug::CONV_N2) : -1;
     l.off_park_flags = parks ? take(sizeof(int) * (int64_t)aug::PARK_SMS * aug::PARK_PER_SM) : -1;
     l.off_ys = take(sizeof(float) * B * l.ws_stride);
     l.off_vv = take(sizeof(float) * B * l.ws_stride);
     l.off_energy = take(sizeof(double) * 2 * B);
-    l.off_leff = take(sizeof(int) * B);
+    l.off_leff = take(sizeof(int) * (B + 1));
     l.off_gain = take(sizeof(float) * B);
     l.off_melw = take(sizeof(aug::MelBin) * B * l.n_bins);
     l.off_melstart = take(sizeof(int) * B * (c.n_mel + 2));
@@ -254,6 +254,16 @@ int aug_create(AugCtx **out, const AugConfig *cfg, void *cuda_stream) {
         ctx->st_feats = reinterpret_cast<float *>(base + l.off_st_feats);
         ctx->st_counts = reinterpret_cast<int *>(base + l.off_st_counts);
     }
+    if (ctx->route == aug::ROUTE_STORED) {
+        if (cudaHostAlloc(reinterpret_cast<void **>(&ctx->leff_seen), sizeof(int), cudaHostAllocDefault) !=
+            cudaSuccess) {
+            cudaGetLastError();
+            cudaFree(ctx->ws_base);
+            delete ctx;
+            return AUG_ENOMEM;
+        }
+        *ctx->leff_seen = 0;
+    }
     if (cfg->host_staging) {
         bool ok_s = cudaStreamCreateWithFlags(&ctx->s_h2d, cudaStreamNonBlocking) == cudaSuccess &&
                     cudaStreamCreateWithFlags(&ctx->s_d2h, cudaStreamNonBlocking) == cudaSuccess &&
@@ -262,6 +272,7 @@ int aug_create(AugCtx **out, const AugConfig *cfg, void *cuda_stream) {
             ok_s = cudaEventCreateWithFlags(&ctx->ev_in[i], cudaEventDisableTiming) == cudaSuccess &&
                    cudaEventCreateWithFlags(&ctx->ev_out[i], cudaEventDisableTiming) == cudaSuccess;
         if (!ok_s) {
+            if (ctx->leff_seen) cudaFreeHost(ctx->leff_seen);
             cudaFree(ctx->ws_base);
             delete ctx;
             return AUG_ECUDA;
@@ -280,6 +291,7 @@ int aug_create(AugCtx **out, const AugConfig *cfg, void *cuda_stream) {
     if (ctx->park_flags &&
         cudaMemsetAsync(ctx->park_flags, 0, sizeof(int) * aug::PARK_SMS * aug::PARK_PER_SM, ctx->stream) !=
             cudaSuccess) {
+        if (ctx->leff_seen) cudaFreeHost(ctx->leff_seen);
         cudaFree(ctx->ws_base);
         delete ctx;
         return AUG_ECUDA;
@@ -290,6 +302,7 @@ int aug_create(AugCtx **out, const AugConfig *cfg, void *cuda_stream) {
                               ctx->stream) == cudaSuccess &&
               cudaStreamSynchronize(ctx->stream) == cudaSuccess;
     if (!ok) {
+        if (ctx->leff_seen) cudaFreeHost(ctx->leff_seen);
         cudaFree(ctx->ws_base);
         delete ctx;
         return AUG_ECUDA;
@@ -318,6 +331,7 @@ int aug_destroy(AugCtx *ctx) {
         cudaStreamDestroy(ctx->s_h2d);
         cudaStreamDestroy(ctx->s_d2h);
     }
+    if (ctx->leff_seen) cudaFreeHost(ctx->leff_seen);
     if (cudaFree(ctx->ws_base) != cudaSuccess) rc = AUG_ECUDA;
     delete ctx;
     return rc;

@@ -68,7 +68,9 @@ struct AugCtx {
     float *ys;             // [max_batch][ws_stride]
     float *vv;             // [max_batch][ws_stride]
     double *energy;        // [max_batch][2]
-    int *leff;             // [max_batch] taps up to the last non-zero one, largest over the utterance's sources
+    int *leff;             // [max_batch + 1] (last entry: largest over the batch)
+    int *leff_seen;        // pinned host copy of that last entry from an earlier call (long-response contexts)
+    int stored_only;       // this call launches the stored-spectra kernels alone taps up to the last non-zero one, largest over the utterance's sources
     float *gain;           // [max_batch] noise gain g for the requested SNR
     aug::MelBin *melw;     // [max_batch][n_bins]
     int *melstart;         // [max_batch][n_mel + 2]

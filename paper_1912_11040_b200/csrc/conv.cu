@@ -26,7 +26,16 @@
 // utterance, the number of taps up to the last non-zero one (the largest over its
 // sources); the fused route then takes 16384 - that + 1 outputs from every block
 // instead of 16384 - rir_taps + 1, and the stored-spectra route skips the partitions
-// that are zero throughout.  The result is the same convolution.
+// that are zero throughout.  A context sized for long responses sends a batch whose
+// responses all end within 8192 taps through the fused route as well: the kernels of
+// both routes are launched, look at the batch's largest effective length first, and
+// those of the route not taken return at once.  The largest effective length of a batch
+// is also copied to the host without waiting for it; while the last value seen says
+// "long", the next call launches the stored-spectra kernels alone (they serve any
+// length), so a stream of long-response batches pays nothing for the choice.  (Routing
+// utterance by utterance was
+// measured too: a minority of long CTAs of the fused kernel beside the stored-spectra
+// kernels balanced badly.)  The result is the same convolution.
 //
 // A real transform of F points is a complex transform of F/2 points on (even, odd)
 // sample pairs followed by the usual split; in the 8192-point routes thread t owns
@@ -227,27 +236,56 @@ __device__ __forceinline__ void finish_block(const float2 (*acc)[2], float2 *sm,
     __syncthreads();
 }
 
-// Largest (index + 1) of a non-zero tap seen by the CTA -> leff[utt] (atomic maximum).
-__device__ __forceinline__ void record_length(int last_plus_1, int *leff_slot, int *red_i, int t) {
+// Effective length of the responses: (index + 1) of the last non-zero tap, largest over the
+// sources of an utterance (leff[utt]) and over the batch (*leff_all); both zeroed before the launch.
+__global__ void __launch_bounds__(CT)
+rir_length_kernel(const float *__restrict__ rir, const AugUttParams *__restrict__ table, int S_max, int L,
+                  int *__restrict__ leff, int *__restrict__ leff_all) {
+    __shared__ int red_i[CT / 32];
+    const int s = blockIdx.x, utt = blockIdx.y, t = threadIdx.x;
+    const AugUttParams &row = table[utt];
+    if (row.n_src < 1 || row.n_src > S_max || s >= row.n_src) return;
+    const float *h = rir + ((int64_t)utt * S_max + s) * L;
+    int last = 0;
+    if ((reinterpret_cast<uintptr_t>(h) & 15) == 0) {
+        for (int i = 4 * t; i + 3 < L; i += 4 * CT) {
+            const float4 z = __ldg(reinterpret_cast<const float4 *>(h + i));
+            if (z.x != 0.f) last = i + 1;
+            if (z.y != 0.f) last = i + 2;
+            if (z.z != 0.f) last = i + 3;
+            if (z.w != 0.f) last = i + 4;
+        }
+        for (int i = (L & ~3) + t; i < L; i += CT)
+            if (h[i] != 0.f) last = max(last, i + 1);
+    } else {
+        for (int i = t; i < L; i += CT)
+            if (h[i] != 0.f) last = i + 1;
+    }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) last_plus_1 = max(last_plus_1, __shfl_xor_sync(0xffffffffu, last_plus_1, o));
-    if ((t & 31) == 0) red_i[t >> 5] = last_plus_1;
+    for (int o = 16; o > 0; o >>= 1) last = max(last, __shfl_xor_sync(0xffffffffu, last, o));
+    if ((t & 31) == 0) red_i[t >> 5] = last;
     __syncthreads();
     if (t == 0) {
         int m = 0;
         for (int i = 0; i < CT / 32; ++i) m = max(m, red_i[i]);
-        if (m > 0) atomicMax(leff_slot, m);
+        if (m > 0) {
+            atomicMax(&leff[utt], m);
+            atomicMax(leff_all, m);
+        }
     }
 }
+
+// Which route a batch takes in a context sized for responses of more than 8192 taps.
+__device__ __forceinline__ bool takes_fused_route(int leff_batch) { return leff_batch <= 2 * BLK; }
 
 // ---------------------------------------------------------------- partition spectra
 __global__ void __launch_bounds__(CT)
 rir_spectra_kernel(const float *__restrict__ rir, const AugUttParams *__restrict__ table, int S_max,
                    int L, int P, const float2 *__restrict__ tw, float2 *__restrict__ hspec,
-                   int *__restrict__ leff) {
+                   const int *__restrict__ leff_all, int always) {
     extern __shared__ __align__(16) float2 sm[];
-    __shared__ int red_i[CT / 32];
     const int p = blockIdx.x, s = blockIdx.y, utt = blockIdx.z, t = threadIdx.x;
+    if (!always && takes_fused_route(*leff_all)) return;
     const AugUttParams &row = table[utt];
     if (row.n_src < 1 || row.n_src > S_max || s >= row.n_src) return;
     const float scale = (s == 0 ? 1.f : row.noise_weight[s - 1]) / (float)aug::CONV_F;
@@ -255,7 +293,6 @@ rir_spectra_kernel(const float *__restrict__ rir, const AugUttParams *__restrict
     float2 *out = hspec + (((int64_t)utt * S_max + s) * P + p) * N2;
 
     float2 v[1][E];
-    int last = 0;
 #pragma unroll
     for (int r = 0; r < E; ++r) {
         const int n = t + CT * r;                 // complex index; taps 2n, 2n+1 of the partition
@@ -264,12 +301,9 @@ rir_spectra_kernel(const float *__restrict__ rir, const AugUttParams *__restrict
         if (n < BLK / 2) {
             if (i0 < L) z.x = h[i0];
             if (i0 + 1 < L) z.y = h[i0 + 1];
-            if (z.x != 0.f) last = max(last, i0 + 1);
-            if (z.y != 0.f) last = max(last, i0 + 2);
         }
         v[0][r] = z;
     }
-    record_length(last, &leff[utt], red_i, t);
     fft4096_from_regs(v, sm, t, tw);
 #pragma unroll
     for (int q = 0; q < NQ; ++q) {
@@ -288,11 +322,11 @@ block_spectra_kernel(const float *__restrict__ speech, int64_t stride,
                      const int *__restrict__ lengths, const float *__restrict__ bank,
                      int64_t bank_len, const AugUttParams *__restrict__ table, int S_max,
                      const float2 *__restrict__ tw, float2 *__restrict__ xspec, int nblk_cap,
-                     int *status, int n_cap) {
+                     int *status, int n_cap, const int *__restrict__ leff_all, int always) {
     extern __shared__ __align__(16) float2 sm[];
     const int b = blockIdx.x, s = blockIdx.y, utt = blockIdx.z, t = threadIdx.x;
     const int N = min(max(lengths[utt], 0), n_cap);
-    if ((int64_t)b * BLK >= N) return;
+    if ((int64_t)b * BLK >= N || (!always && takes_fused_route(*leff_all))) return;
     const AugUttParams &row = table[utt];
     if (row.n_src < 1 || row.n_src > S_max || s >= row.n_src) return;
     const float *x;
@@ -321,14 +355,15 @@ spectral_convolve_kernel(const int *__restrict__ lengths, const float *__restric
                          const float2 *__restrict__ hspec, const float2 *__restrict__ xspec,
                          int nblk_cap, const float2 *__restrict__ tw, float *__restrict__ ys,
                          float *__restrict__ vv, int64_t ws_stride, double *__restrict__ energy,
-                         int n_cap, const int *__restrict__ leff) {
+                         int n_cap, const int *__restrict__ leff, const int *__restrict__ leff_all,
+                         int always) {
     extern __shared__ __align__(16) float2 sm[];
     __shared__ float red[CT / 32];
     const int b = blockIdx.x, utt = blockIdx.y, t = threadIdx.x;
     // partitions behind the last non-zero tap of every source of this utterance are zero
     const int P_used = min(P, (max(leff[utt], 1) + BLK - 1) / BLK);
     const int N = min(max(lengths[utt], 0), n_cap);
-    if ((int64_t)b * BLK >= N) return;
+    if ((int64_t)b * BLK >= N || (!always && takes_fused_route(*leff_all))) return;
     const AugUttParams &row = table[utt];
     int n_src = row.n_src;
     if (n_src < 1 || n_src > S_max) n_src = 0;
@@ -626,17 +661,20 @@ __device__ __forceinline__ void edge_inverse(const Edge &y, float2 uh, float2 &a
 // the whole second half are zero), scaled by the noise weight and 1/F.
 __global__ void __launch_bounds__(CT)
 rir_spectra2_kernel(const float *__restrict__ rir, const AugUttParams *__restrict__ table, int S_max,
-                    int L, const float2 *__restrict__ tw, float2 *__restrict__ hspec,
-                    int *__restrict__ leff) {
+                    int L, const float2 *__restrict__ tw, float2 *__restrict__ hspec, int64_t hs_stride,
+                    const int *__restrict__ leff, const int *__restrict__ leff_all, int mixed) {
     extern __shared__ __align__(16) float2 sm[];
     __shared__ int red_i[CT / 32];
     float2 *A = sm, *Bf = sm + SM_POINTS;
     const int s = blockIdx.x, utt = blockIdx.y, t = threadIdx.x;
+    // mixed: the lengths are known already (rir_length_kernel) and decide the route; otherwise
+    // this kernel reads every tap anyway and records the length on the way
+    if (mixed && !takes_fused_route(*leff_all)) return;
     const AugUttParams &row = table[utt];
     if (row.n_src < 1 || row.n_src > S_max || s >= row.n_src) return;
     const float scale = (s == 0 ? 1.f : row.noise_weight[s - 1]) / (float)F2;
     const float *h = rir + ((int64_t)utt * S_max + s) * L;
-    float2 *out = hspec + ((int64_t)utt * S_max + s) * NB2;
+    float2 *out = hspec + ((int64_t)utt * S_max + s) * hs_stride;
     {
         float2 va[1][E], vb[1][E];
         int last = 0;
@@ -649,15 +687,25 @@ rir_spectra2_kernel(const float *__restrict__ rir, const AugUttParams *__restric
                 if (i0 + 1 < L) z.y = h[i0 + 1];
                 if (i0 + 2 < L) z.z = h[i0 + 2];
                 if (i0 + 3 < L) z.w = h[i0 + 3];
-                if (z.x != 0.f) last = max(last, i0 + 1);
-                if (z.y != 0.f) last = max(last, i0 + 2);
-                if (z.z != 0.f) last = max(last, i0 + 3);
-                if (z.w != 0.f) last = max(last, i0 + 4);
+                if (z.x != 0.f) last = i0 + 1;
+                if (z.y != 0.f) last = i0 + 2;
+                if (z.z != 0.f) last = i0 + 3;
+                if (z.w != 0.f) last = i0 + 4;
             }
             va[0][r] = make_float2(z.x, z.y);
             vb[0][r] = make_float2(z.z, z.w);
         }
-        record_length(last, &leff[utt], red_i, t);
+        if (!mixed) {
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) last = max(last, __shfl_xor_sync(0xffffffffu, last, o));
+            if ((t & 31) == 0) red_i[t >> 5] = last;
+            __syncthreads();
+            if (t == 0) {
+                int m = 0;
+                for (int i = 0; i < CT / 32; ++i) m = max(m, red_i[i]);
+                if (m > 0) atomicMax(const_cast<int *>(&leff[utt]), m);
+            }
+        }
         fft2x4096_from_regs(va, vb, A, Bf, t, tw);
         __syncthreads();
     }
@@ -711,7 +759,9 @@ convolve_fused2_kernel(const float *__restrict__ speech, int64_t stride,
                        const float2 *__restrict__ hspec, const float2 *__restrict__ tw,
                        float *__restrict__ ys, float *__restrict__ vv, int64_t ws_stride,
                        double *__restrict__ energy, int *status, int n_cap,
-                       const int *__restrict__ leff, float2 *__restrict__ park, int *park_flags, int n_sm) {
+                       const int *__restrict__ leff, const int *__restrict__ leff_all, int64_t hs_stride,
+                       int mixed,
+                       float2 *__restrict__ park, int *park_flags, int n_sm) {
     extern __shared__ __align__(16) float2 sm[];
     float2 *A = sm, *Bf = sm + SM_POINTS;
     __shared__ float red[CT / 32];
@@ -720,7 +770,9 @@ convolve_fused2_kernel(const float *__restrict__ speech, int64_t stride,
     const int N = min(max(lengths[utt], 0), n_cap);
     // every block yields the F2 - (taps - 1) outputs that see no wrap-around, cut to a multiple
     // of 4, where taps counts up to the last non-zero tap of this utterance's responses
-    const int ob = (F2 - min(max(leff[utt], 1), BLK2) + 1) & ~3;
+    if (mixed && !takes_fused_route(*leff_all)) return;
+    const int taps_used = leff[utt];
+    const int ob = (F2 - min(max(taps_used, 1), BLK2) + 1) & ~3;
     if ((int64_t)b * ob >= N) return;
     const AugUttParams &row = table[utt];
     int n_src = row.n_src;
@@ -771,7 +823,7 @@ convolve_fused2_kernel(const float *__restrict__ speech, int64_t stride,
             load_segment4(va, vb, x, s != 0, nlen, (b + 1) * ob - F2, N, t, bank + bank_len);
             fft2x4096_from_regs(va, vb, A, Bf, t, tw);
         }
-        const float2 *H = hspec + ((int64_t)utt * S_max + s) * NB2;
+        const float2 *H = hspec + ((int64_t)utt * S_max + s) * hs_stride;
         // the first slot's operands are requested before the barrier that completes the transform
         SpecOps nxt = load_spec_ops(H, tw, t);
         __syncthreads();
@@ -897,26 +949,43 @@ constexpr size_t FFT2_SMEM = 2 * FFT_SMEM;
 
 }  // namespace
 
+static bool stored_route(const AugCtx *ctx) { return ctx->route == aug::ROUTE_STORED; }
+// response spectra of one (utterance, source): complex numbers between consecutive ones
+static int64_t hspec_stride(const AugCtx *ctx) { return stored_route(ctx) ? (int64_t)ctx->n_part * N2 : NB2; }
+
 int launch_rir_spectra(AugCtx *ctx, const float *rir, const AugUttParams *table, int B,
                        cudaStream_t st) {
     const AugConfig &c = ctx->cfg;
+    const int mixed = stored_route(ctx) ? 1 : 0;
+    // long-response context: the last batch size seen decides whether the fused kernels are launched at all
+    ctx->stored_only = mixed && ctx->leff_seen && *ctx->leff_seen > BLK2;
+    int *leff_all = ctx->leff + ctx->cfg.max_batch;
     AUG_CUDA_OK(cudaMemsetAsync(ctx->leff, 0, sizeof(int) * (size_t)B, st));
-    if (ctx->route == aug::ROUTE_FUSED_8192) {
+    AUG_CUDA_OK(cudaMemsetAsync(leff_all, 0, sizeof(int), st));
+    dim3 grid2(c.max_sources, B);
+    if (mixed) {
+        rir_length_kernel<<<grid2, CT, 0, st>>>(rir, table, c.max_sources, c.rir_taps, ctx->leff, leff_all);
+        AUG_CUDA_OK(cudaGetLastError());
+        ctx->launches++;
+    }
+    if (!ctx->stored_only) {
         if (smem_opt_in<rir_spectra2_kernel>(ctx->device) != AUG_OK) return AUG_ECUDA;
-        dim3 grid(c.max_sources, B);
-        rir_spectra2_kernel<<<grid, CT, FFT2_SMEM, st>>>(rir, table, c.max_sources, c.rir_taps, ctx->tw,
-                                                         ctx->hspec, ctx->leff);
-    } else {
+        rir_spectra2_kernel<<<grid2, CT, FFT2_SMEM, st>>>(rir, table, c.max_sources, c.rir_taps, ctx->tw,
+                                                          ctx->hspec, hspec_stride(ctx), ctx->leff, leff_all,
+                                                          mixed);
+        AUG_CUDA_OK(cudaGetLastError());
+        ctx->launches++;
+    }
+    if (mixed) {
         dim3 grid(ctx->n_part, c.max_sources, B);
         rir_spectra_kernel<<<grid, CT, FFT_SMEM, st>>>(rir, table, c.max_sources, c.rir_taps,
-                                                       ctx->n_part, ctx->tw, ctx->hspec, ctx->leff);
+                                                       ctx->n_part, ctx->tw, ctx->hspec, leff_all,
+                                                       ctx->stored_only);
+        AUG_CUDA_OK(cudaGetLastError());
+        ctx->launches++;
     }
-    AUG_CUDA_OK(cudaGetLastError());
-    ctx->launches++;
     return AUG_OK;
 }
-
-static bool stored_route(const AugCtx *ctx) { return ctx->route == aug::ROUTE_STORED; }
 
 int launch_convolve_prepare(AugCtx *ctx, const float *speech, int64_t stride, const int *lengths,
                             const float *bank, int64_t bank_len, const AugUttParams *table, int B,
@@ -929,7 +998,7 @@ int launch_convolve_prepare(AugCtx *ctx, const float *speech, int64_t stride, co
     dim3 grid_x(nblk, c.max_sources, B);
     block_spectra_kernel<<<grid_x, CT, FFT_SMEM, ctx->stream>>>(
         speech, stride, lengths, bank, bank_len, table, c.max_sources, ctx->tw, ctx->xspec,
-        ctx->nblk_cap, ctx->status, max_len);
+        ctx->nblk_cap, ctx->status, max_len, ctx->leff + c.max_batch, ctx->stored_only);
     AUG_CUDA_OK(cudaGetLastError());
     ctx->launches++;
     return AUG_OK;
@@ -940,11 +1009,12 @@ int launch_convolve_finish(AugCtx *ctx, const float *speech, int64_t stride, con
                            int max_len) {
     const AugConfig &c = ctx->cfg;
     if (max_len <= 0) return AUG_OK;
-    const int nblk = (max_len + BLK - 1) / BLK;
-    dim3 grid(nblk, B);
-    if (ctx->route == aug::ROUTE_FUSED_8192) {
-        // the grid covers the shortest block any utterance can have (a response that fills its buffer)
-        const int ob_min = (F2 - c.rir_taps + 1) & ~3;
+    const int mixed = stored_route(ctx) ? 1 : 0;
+    const int *leff_all = ctx->leff + c.max_batch;
+    if (!ctx->stored_only) {
+        // fused route: the grid covers the shortest block an utterance on it can have (a response
+        // that fills min(rir_taps, 8192) taps)
+        const int ob_min = (F2 - min(c.rir_taps, BLK2) + 1) & ~3;
         const int nblk2 = (max_len + ob_min - 1) / ob_min;
         dim3 grid2(nblk2, B);
         auto kern = ctx->park ? convolve_fused2_kernel<true> : convolve_fused2_kernel<false>;
@@ -953,15 +1023,24 @@ int launch_convolve_finish(AugCtx *ctx, const float *speech, int64_t stride, con
             return AUG_ECUDA;
         kern<<<grid2, CT, FFT2_SMEM, ctx->stream>>>(
             speech, stride, lengths, bank, bank_len, table, c.max_sources, ctx->hspec, ctx->tw,
-            ctx->ys, ctx->vv, ctx->ws_stride, ctx->energy, ctx->status, max_len, ctx->leff, ctx->park,
-            ctx->park_flags, ctx->n_sm);
-    } else {
+            ctx->ys, ctx->vv, ctx->ws_stride, ctx->energy, ctx->status, max_len, ctx->leff, leff_all,
+            hspec_stride(ctx), mixed, ctx->park, ctx->park_flags, ctx->n_sm);
+        AUG_CUDA_OK(cudaGetLastError());
+        ctx->launches++;
+    }
+    if (mixed) {
+        const int nblk = (max_len + BLK - 1) / BLK;
+        dim3 grid(nblk, B);
         spectral_convolve_kernel<<<grid, CT, FFT_SMEM, ctx->stream>>>(
             lengths, bank, bank_len, table, c.max_sources, ctx->n_part, ctx->hspec, ctx->xspec,
-            ctx->nblk_cap, ctx->tw, ctx->ys, ctx->vv, ctx->ws_stride, ctx->energy, max_len, ctx->leff);
+            ctx->nblk_cap, ctx->tw, ctx->ys, ctx->vv, ctx->ws_stride, ctx->energy, max_len, ctx->leff, leff_all,
+            ctx->stored_only);
+        AUG_CUDA_OK(cudaGetLastError());
+        ctx->launches++;
+        // for the next call's choice (not waited for)
+        if (ctx->leff_seen)
+            AUG_CUDA_OK(cudaMemcpyAsync(ctx->leff_seen, leff_all, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
     }
-    AUG_CUDA_OK(cudaGetLastError());
-    ctx->launches++;
     snr_gain_kernel<<<(B + 255) / 256, 256, 0, ctx->stream>>>(ctx->energy, table, B, ctx->gain);
     AUG_CUDA_OK(cudaGetLastError());
     ctx->launches++;
