@@ -81,7 +81,7 @@ struct Layout {
     int64_t ws_stride;
     int64_t off_xspec, off_park, off_park_flags;
     int64_t off_tw, off_rir, off_hspec, off_ys, off_vv, off_energy, off_leff, off_gain, off_melw, off_melstart,
-        off_status, off_warped, off_st_speech, off_st_bank, off_st_table, off_st_lengths,
+        off_status, off_warped, off_vtlp_tab, off_st_speech, off_st_bank, off_st_table, off_st_lengths,
         off_st_feats, off_st_counts, total;
 };
 
@@ -113,6 +113,7 @@ Layout make_layout(const AugConfig &c) {
     l.off_melstart = take(sizeof(int) * B * (c.n_mel + 2));
     l.off_status = take(sizeof(int) * 2);
     l.off_warped = c.vtlp_win > 0 ? take(sizeof(float) * B * l.ws_stride) : -1;
+    l.off_vtlp_tab = c.vtlp_win > 0 ? take((sizeof(int) + sizeof(float)) * B * 513) : -1;
     if (c.host_staging) {
         l.off_st_speech = take(sizeof(float) * B * l.ws_stride);
         l.off_st_bank = take(sizeof(float) * (c.max_bank_samples > 0 ? c.max_bank_samples : 1));
@@ -246,6 +247,7 @@ int aug_create(AugCtx **out, const AugConfig *cfg, void *cuda_stream) {
     ctx->melstart = reinterpret_cast<int *>(base + l.off_melstart);
     ctx->status = reinterpret_cast<int *>(base + l.off_status);
     ctx->warped = l.off_warped >= 0 ? reinterpret_cast<float *>(base + l.off_warped) : nullptr;
+    ctx->vtlp_tab = l.off_vtlp_tab >= 0 ? base + l.off_vtlp_tab : nullptr;
     if (cfg->host_staging) {
         ctx->st_speech = reinterpret_cast<float *>(base + l.off_st_speech);
         ctx->st_bank = reinterpret_cast<float *>(base + l.off_st_bank);

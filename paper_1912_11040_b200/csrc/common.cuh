@@ -65,6 +65,7 @@ struct AugCtx {
     int *park_flags;       // [PARK_SMS * PARK_PER_SM] 1 = slot taken
     int n_sm;              // multiprocessors with slots (PARK_SMS); CTAs on others sum in the time domain
     float *warped;         // [max_batch][ws_stride] speech after the waveform warp; NULL unless cfg.vtlp_win
+    void *vtlp_tab;        // [max_batch][513] lower source bin (int), then [max_batch][513] fraction (float)
     float *ys;             // [max_batch][ws_stride]
     float *vv;             // [max_batch][ws_stride]
     double *energy;        // [max_batch][2]

@@ -14,7 +14,9 @@
 // directly (bin k from Z around k0, bin K-k from Z around K-k0), and the inverse of
 // the packed spectrum returns the two frames in its real and imaginary part.
 // A CTA owns the output samples of HB hops and computes the HB + 3 frames that
-// cover them, so nothing is added across CTAs.
+// cover them, so nothing is added across CTAs: four 64-thread groups transform a
+// frame pair each, then every thread adds what the round's frames contribute to the
+// output samples it owns (in registers), and so on for the next round.
 #include "common.cuh"
 #include "fft.cuh"
 
@@ -24,17 +26,16 @@ using namespace augfft;
 constexpr int K = 1024;
 constexpr int E = 16;                 // points per thread
 constexpr int GROUP = K / E;          // 64 threads per transform
-constexpr int NGROUP = 2;
+constexpr int NGROUP = 4;
 constexpr int RS_THREADS = GROUP * NGROUP;
-constexpr int HB = 8;                 // hops of output per CTA
+constexpr int HB = 16;                // hops of output per CTA
 constexpr int NF = HB + 3;            // frames that cover them
 constexpr int XB = padded_points(K);
 
 __host__ __device__ constexpr size_t resynth_smem(int win) {
     const int hop = win / 4;
     return sizeof(float2) * 2 * NGROUP * XB + sizeof(float) * (size_t)((NF - 1) * hop + win) +
-           sizeof(float) * (size_t)NF * win + sizeof(float) * win + sizeof(float) * (K / 2 + 1) +
-           sizeof(int) * (K / 2 + 1);
+           sizeof(float) * win + sizeof(float) * (K / 2 + 1) + sizeof(int) * (K / 2 + 1);
 }
 
 __device__ __forceinline__ void fft1024_from_regs(float2 (*v)[E], float2 *s, int tg, const float2 *__restrict__ tw,
@@ -50,17 +51,37 @@ __device__ __forceinline__ void fft1024_in_place(float2 *s, int tg, const float2
     pass<K, E, 8, 128, 16>(s, tg, tw, gsync);
 }
 
+// Source position of every bin of an utterance: the frequency that Eq. 1 moves to bin k, in
+// bins, as lower bin and fraction (fp64: a position error of 6e-5 bins, one fp32 ulp at bin 512,
+// would already cost half of the waveform tolerance).
+__global__ void __launch_bounds__(256)
+vtlp_positions_kernel(const AugUttParams *__restrict__ table, int *__restrict__ k0_tab,
+                      float *__restrict__ fr_tab) {
+    const int utt = blockIdx.x;
+    const double a = 1.0 - (double)table[utt].alpha;
+    const double PI = 3.14159265358979323846;
+    for (int k = threadIdx.x; k <= K / 2; k += 256) {
+        const double om = 2.0 * PI * k / K;
+        double pos = (om - 2.0 * atan(a * sin(om) / (1.0 + a * cos(om)))) * K / (2.0 * PI);
+        if (k == 0) pos = 0.0;
+        if (k == K / 2) pos = (double)(K / 2);
+        int k0 = (int)floor(pos);
+        k0 = min(max(k0, 0), K / 2 - 1);
+        k0_tab[(int64_t)utt * (K / 2 + 1) + k] = k0;
+        fr_tab[(int64_t)utt * (K / 2 + 1) + k] = (float)(pos - (double)k0);
+    }
+}
+
 __global__ void __launch_bounds__(RS_THREADS)
 vtlp_resynth_kernel(const float *__restrict__ speech, int64_t stride, const int *__restrict__ lengths,
-                    const AugUttParams *__restrict__ table, int win, const float2 *__restrict__ tw,
-                    float *__restrict__ out, int64_t out_stride, int n_cap) {
+                    const int *__restrict__ k0_tab, const float *__restrict__ fr_tab, int win,
+                    const float2 *__restrict__ tw, float *__restrict__ out, int64_t out_stride, int n_cap) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int hop = win >> 2, front = win - hop;
     float2 *zbuf = reinterpret_cast<float2 *>(smem_raw);            // [NGROUP][XB] forward transforms
     float2 *wbuf = zbuf + NGROUP * XB;                              // [NGROUP][XB] warped spectra / inverse
     float *xin = reinterpret_cast<float *>(wbuf + NGROUP * XB);     // [(NF-1) hop + win] padded input stretch
-    float *fout = xin + (NF - 1) * hop + win;                       // [NF][win] resynthesised, windowed frames
-    float *wn = fout + NF * win;                                    // [win] Hann
+    float *wn = xin + (NF - 1) * hop + win;                         // [win] Hann
     float *fr_s = wn + win;                                         // [K/2+1] interpolation fraction
     int *k0_s = reinterpret_cast<int *>(fr_s + K / 2 + 1);          // [K/2+1] lower source bin
 
@@ -73,20 +94,9 @@ vtlp_resynth_kernel(const float *__restrict__ speech, int64_t stride, const int 
     const float *x = speech + (int64_t)utt * stride;
     float *y = out + (int64_t)utt * out_stride;
 
-    // source position of every bin: the frequency Eq. 1 moves to bin k, in bins
-    {
-        const double a = 1.0 - (double)table[utt].alpha;
-        const double PI = 3.14159265358979323846;
-        for (int k = tid; k <= K / 2; k += RS_THREADS) {
-            const double om = 2.0 * PI * k / K;
-            double pos = (om - 2.0 * atan(a * sin(om) / (1.0 + a * cos(om)))) * K / (2.0 * PI);
-            if (k == 0) pos = 0.0;
-            if (k == K / 2) pos = (double)(K / 2);
-            int k0 = (int)floor(pos);
-            k0 = min(max(k0, 0), K / 2 - 1);
-            k0_s[k] = k0;
-            fr_s[k] = (float)(pos - (double)k0);
-        }
+    for (int k = tid; k <= K / 2; k += RS_THREADS) {
+        k0_s[k] = k0_tab[(int64_t)utt * (K / 2 + 1) + k];
+        fr_s[k] = fr_tab[(int64_t)utt * (K / 2 + 1) + k];
     }
     for (int n = tid; n < win; n += RS_THREADS) wn[n] = 0.5f - 0.5f * cospif(2.f * (float)n / (float)win);
     // input stretch of frames t0-3 .. t0+HB-1 in padded coordinates
@@ -99,67 +109,93 @@ vtlp_resynth_kernel(const float *__restrict__ speech, int64_t stride, const int 
 
     float2 *Z = zbuf + grp * XB, *W = wbuf + grp * XB;
     const GroupSync gsync{grp + 1, GROUP};
-    for (int pr = grp; 2 * pr < NF; pr += NGROUP) {
-        const int fa = 2 * pr, fb = fa + 1;                       // frame slots; frame number = t0 - 3 + slot
-        const bool have_a = t0 - 3 + fa >= 0 && t0 - 3 + fa < T;
-        const bool have_b = fb < NF && t0 - 3 + fb >= 0 && t0 - 3 + fb < T;
-        if (!have_a && !have_b) continue;                         // (uniform over the group)
-        {
-            float2 v[1][E];
+    constexpr int NPAIR = (NF + 1) / 2;
+    constexpr int OWN = (HB * 256 + RS_THREADS - 1) / RS_THREADS;   // owned samples per thread (hop <= 256)
+    float acc[OWN];
 #pragma unroll
-            for (int r = 0; r < E; ++r) {
-                const int n = tg + GROUP * r;
-                float a = 0.f, b = 0.f;
-                if (n < win) {
-                    const float w = wn[n];
-                    if (have_a) a = w * xin[fa * hop + n];
-                    if (have_b) b = w * xin[fb * hop + n];
-                }
-                v[0][r] = make_float2(a, b);
-            }
-            fft1024_from_regs(v, Z, tg, tw, gsync);
-        }
-        // warped packed spectrum, real and imaginary parts swapped for the inverse
-        for (int k = tg; k <= K / 2; k += GROUP) {
-            const int k0 = k0_s[k];
-            const float fr = fr_s[k], om = 1.f - fr;
-            const float2 z0 = Z[pad0(k0)], z1 = Z[pad0(k0 + 1)];
-            W[pad0(k)] = make_float2(fmaf(fr, z1.y, om * z0.y), fmaf(fr, z1.x, om * z0.x));
-            if (k > 0 && k < K / 2) {
-                const float2 m0 = Z[pad0((K - k0) & (K - 1))], m1 = Z[pad0(K - k0 - 1)];
-                W[pad0(K - k)] = make_float2(fmaf(fr, m1.y, om * m0.y), fmaf(fr, m1.x, om * m0.x));
-            }
-        }
-        gsync();
-        fft1024_in_place(W, tg, tw, gsync);
-        for (int n = tg; n < win; n += GROUP) {
-            const float2 z = W[pad0(n)];                           // (imaginary, real) of the inverse, times K
-            const float w = wn[n] * (1.f / (float)K);
-            if (have_a) fout[fa * win + n] = w * z.y;
-            if (have_b) fout[fb * win + n] = w * z.x;
-        }
-        gsync();      // the buffers are refilled by the group's next pair
-    }
-    __syncthreads();
+    for (int u = 0; u < OWN; ++u) acc[u] = 0.f;
+    const float inv_k = 1.f / (float)K;
 
-    // owned samples: hops t0 .. t0+HB-1; sample c is covered by frames c/hop - 3 .. c/hop
-    for (int i = tid; i < HB * hop; i += RS_THREADS) {
+    for (int round = 0; round * NGROUP < NPAIR; ++round) {
+        const int pr = round * NGROUP + grp;
+        const int fa = 2 * pr, fb = fa + 1;                       // frame slots; frame number = t0 - 3 + slot
+        const bool have_a = fa < NF && t0 - 3 + fa >= 0 && t0 - 3 + fa < T;
+        const bool have_b = fb < NF && t0 - 3 + fb >= 0 && t0 - 3 + fb < T;
+        if (have_a || have_b) {                                   // (uniform over the group)
+            {
+                float2 v[1][E];
+#pragma unroll
+                for (int r = 0; r < E; ++r) {
+                    const int n = tg + GROUP * r;
+                    float a = 0.f, b = 0.f;
+                    if (n < win) {
+                        const float w = wn[n];
+                        if (have_a) a = w * xin[fa * hop + n];
+                        if (have_b) b = w * xin[fb * hop + n];
+                    }
+                    v[0][r] = make_float2(a, b);
+                }
+                fft1024_from_regs(v, Z, tg, tw, gsync);
+            }
+            // warped packed spectrum, real and imaginary parts swapped for the inverse
+            for (int k = tg; k <= K / 2; k += GROUP) {
+                const int k0 = k0_s[k];
+                const float fr = fr_s[k], om = 1.f - fr;
+                const float2 z0 = Z[pad0(k0)], z1 = Z[pad0(k0 + 1)];
+                W[pad0(k)] = make_float2(fmaf(fr, z1.y, om * z0.y), fmaf(fr, z1.x, om * z0.x));
+                if (k > 0 && k < K / 2) {
+                    const float2 m0 = Z[pad0((K - k0) & (K - 1))], m1 = Z[pad0(K - k0 - 1)];
+                    W[pad0(K - k)] = make_float2(fmaf(fr, m1.y, om * m0.y), fmaf(fr, m1.x, om * m0.x));
+                }
+            }
+            gsync();
+            fft1024_in_place(W, tg, tw, gsync);               // W[n] = (imaginary, real) of the inverse, times K
+        }
+        __syncthreads();
+        // what this round's frames add to the owned samples: sample i of the CTA sits at
+        // n = i + (3 - slot) hop of the frame in `slot`
+#pragma unroll
+        for (int u = 0; u < OWN; ++u) {
+            const int i = tid + u * RS_THREADS;
+            if (i < HB * hop) {
+                float sum = 0.f;
+                for (int g = 0; g < NGROUP; ++g) {
+                    const int slot = 2 * (round * NGROUP + g);
+                    const float2 *Wg = wbuf + g * XB;
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const int sl = slot + h, t = t0 - 3 + sl;
+                        const int n = i + (3 - sl) * hop;
+                        if (sl < NF && t >= 0 && t < T && n >= 0 && n < win) {
+                            const float2 z = Wg[pad0(n)];
+                            sum = fmaf(wn[n], h ? z.x : z.y, sum);
+                        }
+                    }
+                }
+                acc[u] = fmaf(sum, inv_k, acc[u]);
+            }
+        }
+        __syncthreads();      // the buffers are refilled in the next round
+    }
+
+    // owned samples: sample c is covered by frames c/hop - 3 .. c/hop; divide by their squared windows
+#pragma unroll
+    for (int u = 0; u < OWN; ++u) {
+        const int i = tid + u * RS_THREADS;
         const int c = t0 * hop + i;
         const int idx = c - front;
-        if (idx < 0 || idx >= N) continue;
+        if (i >= HB * hop || idx < 0 || idx >= N) continue;
         const int hb = t0 + i / hop;
-        float acc = 0.f, norm = 0.f;
+        float norm = 0.f;
 #pragma unroll
         for (int d = 0; d < 4; ++d) {
             const int t = hb - d;
             if (t >= 0 && t < T) {
-                const int n = c - t * hop;
-                const float w = wn[n];
-                acc += fout[(t - (t0 - 3)) * win + n];
+                const float w = wn[c - t * hop];
                 norm = fmaf(w, w, norm);
             }
         }
-        y[idx] = acc / norm;
+        y[idx] = acc[u] / norm;
     }
 }
 
@@ -173,9 +209,14 @@ int launch_vtlp_resynth(AugCtx *ctx, const float *speech, int64_t stride, const 
     const int T_cap = (max_len + front + hop - 1) / hop;
     const size_t smem = resynth_smem(win);
     if (smem_opt_in<vtlp_resynth_kernel>(ctx->device) != AUG_OK) return AUG_ECUDA;
+    int *k0_tab = reinterpret_cast<int *>(ctx->vtlp_tab);
+    float *fr_tab = reinterpret_cast<float *>(k0_tab + (size_t)ctx->cfg.max_batch * (K / 2 + 1));
+    vtlp_positions_kernel<<<B, 256, 0, ctx->stream>>>(table, k0_tab, fr_tab);
+    AUG_CUDA_OK(cudaGetLastError());
+    ctx->launches++;
     dim3 grid((T_cap + HB - 1) / HB, B);
-    vtlp_resynth_kernel<<<grid, RS_THREADS, smem, ctx->stream>>>(speech, stride, lengths, table, win, ctx->tw,
-                                                                out, out_stride, max_len);
+    vtlp_resynth_kernel<<<grid, RS_THREADS, smem, ctx->stream>>>(speech, stride, lengths, k0_tab, fr_tab, win,
+                                                                ctx->tw, out, out_stride, max_len);
     AUG_CUDA_OK(cudaGetLastError());
     ctx->launches++;
     return AUG_OK;
