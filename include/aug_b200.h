@@ -216,7 +216,9 @@ int aug_rir_image_method(AugCtx *ctx, const AugUttParams *table_dev, int B, floa
  *   wave_out_dev [B][speech_stride] fp32: samples [0,lengths[b]) written,
  *               the rest of each row left untouched
  * y_s = speech * rir[0] and v = sum_k weight_k (noise_k * rir[k]) are causal
- * convolutions cut to the utterance length, done as FFT overlap convolution;
+ * convolutions cut to the utterance length, done as FFT overlap convolution (the
+ * block size follows the last non-zero tap of an utterance's responses, so zero
+ * tails of the response buffers cost nothing);
  * out = y_s + g v with g = sqrt(sum y_s^2 / (sum v^2 10^(snr_db/10))), g = 0 when
  * there is no noise or either sum is zero. */
 int aug_reverb_mix(AugCtx *ctx, const float *speech_dev, int64_t speech_stride,
@@ -342,8 +344,9 @@ int aug_upload_noise_bank(AugCtx *ctx, const float *noise_bank_host, int64_t ban
 /* -------------------------------------------------------------- measurement utilities
  * (instrumentation of this library; the paper has no counterpart) */
 
-#define AUG_N_STAGES 7 /* 0 impulse responses, 1 partition spectra, 2 filterbank tables,
-                          3 block spectra of the audio (multi-partition responses only),
+#define AUG_N_STAGES 7 /* 0 impulse responses, 1 response lengths and spectra, 2 filterbank tables,
+                          3 waveform warp (vtlp_win > 0) and block spectra of the audio (contexts
+                            sized for responses of more than 8192 taps),
                           4 convolution, 5 waveform mix (only when requested), 6 features */
 
 /* The fused convolution (responses of up to 8192 taps) sums several noise sources of an

@@ -160,7 +160,10 @@ __device__ __forceinline__ void tile_power(const float *chunk, int nf, int win, 
 #define FEAT_FT_512 32      // frames per CTA tile, 512-point transform
 #endif
 #ifndef FEAT_FT_1024
-#define FEAT_FT_1024 16     // frames per CTA tile, 1024-point transform
+#define FEAT_FT_1024 8      // frames per CTA tile, 1024-point transform (64 KB of shared memory: 3 CTAs/SM)
+#endif
+#ifndef FEAT_TILES_1024
+#define FEAT_TILES_1024 8   // consecutive tiles one CTA works through, 1024-point transform
 #endif
 #ifndef FEAT_TILES
 #define FEAT_TILES 4        // consecutive tiles one CTA works through
@@ -173,7 +176,7 @@ struct Plan<512> {
 };
 template <>
 struct Plan<1024> {
-    static constexpr int E = 16, FT = FEAT_FT_1024, TILES = FEAT_TILES;
+    static constexpr int E = 16, FT = FEAT_FT_1024, TILES = FEAT_TILES_1024;
 };
 
 // Floats of the region that first holds the transform buffers of the four groups and
