@@ -374,6 +374,9 @@ def run_ours(args):
     w = synth.make_workload(args.workload, seed=rank, batch=args.batch, noise_align=args.noise_align)
     if args.vtlp_win:
         w.cfg["vtlp_win"] = args.vtlp_win          # warp the speech waveform instead of the filterbank
+    # the host entry point returns the frames of every utterance and its frame count; with
+    # "padded" it also transfers the padding rows up to T_max
+    w.cfg["host_rows"] = 1 if args.host_rows == "valid" else 0
     cfg = binding.make_config(w.cfg, w.B, w.stride, host_staging=True, max_bank_samples=w.bank.size)
     ctx = binding.AugContext(cfg)
     speech = torch.from_numpy(w.speech).cuda()
@@ -563,6 +566,7 @@ def run_ours(args):
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
             "data": "synthetic",
             "config": {"workload": workload_label(args.workload), "batch": w.B, "noise_align": args.noise_align, "vtlp_win": args.vtlp_win,
+                       "host_rows": args.host_rows,
                        "audio_seconds_per_step": w.audio_seconds, "parallelism": f"replicas x{world}",
                        "l2": "inputs larger than L2 (speech + noise bank "
                              f"{(speech.numel() + bank.numel()) * 4 / 1e6:.0f} MB per step)"},
@@ -607,6 +611,9 @@ def main():
                     help="utterances given to the numpy/scipy CPU pipeline (0 = skip)")
     ap.add_argument("--noise-align", type=int, default=4, choices=[1, 4],
                     help="noise stretches start and end on multiples of this many samples (1 = anywhere)")
+    ap.add_argument("--host-rows", choices=("valid", "padded"), default="valid",
+                    help="end-to-end leg: feature rows the host call copies back (valid frames only, "
+                         "or all T_max rows of every utterance with their padding)")
     ap.add_argument("--vtlp-win", type=int, default=0,
                     help="apply the warp to the speech waveform with this window (800 = 50 ms) instead of "
                          "inside the filterbank")

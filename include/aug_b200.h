@@ -56,6 +56,14 @@ typedef enum { AUG_COMPRESS_LOG = 0, AUG_COMPRESS_POW_1_15 = 1 } AugCompression;
  * max(|kx|,|ky|,|kz|) <= N, up to 3N reflections: (2N+1)^3 images, a stress mode. */
 typedef enum { AUG_LATTICE_TOTAL = 0, AUG_LATTICE_CUBE = 1 } AugLattice;
 
+/* Rows of the host feature buffer that aug_pipeline_host writes.  PADDED (default): all
+ * T_max rows of every utterance, those at and beyond its frame count holding pad_value.
+ * VALID: only the frame_counts[b] rows that hold features; the other rows of the caller's
+ * buffer are left as they are (a caller that packs by frame count, or keeps a buffer it
+ * filled with its pad value once, saves the transfer of the padding: Section 2.4's
+ * concern is keeping the trainer fed). */
+typedef enum { AUG_HOST_ROWS_PADDED = 0, AUG_HOST_ROWS_VALID = 1 } AugHostRows;
+
 /* Fixed at aug_create.  Plain data, no pointers. */
 typedef struct {
     int32_t fs;              /* sampling rate, Hz */
@@ -82,7 +90,7 @@ typedef struct {
                                 > 0: it is applied to the speech waveform before the simulator,
                                 with this window (samples; a multiple of 4, at most 1024; 800 is
                                 the 50 ms of Section 4) and the filterbank stays unwarped */
-    int32_t reserved_;       /* keeps the struct a multiple of 8 bytes; set to 0 */
+    int32_t host_rows;       /* AugHostRows: what aug_pipeline_host writes to the host feature buffer */
 } AugConfig;
 
 /*
@@ -315,9 +323,13 @@ int aug_pipeline(AugCtx *ctx, const float *speech_dev, int64_t speech_stride,
 
 /* Same call for callers that hold HOST buffers (the context must have been created
  * with host_staging).  Inputs are copied to device staging owned by the context,
- * the path runs, feats (padded, [B][T_max][n_mel]) and frame counts are copied
+ * the path runs, feats ([B][T_max][n_mel]; all rows, padded, or with
+ * AugConfig.host_rows = AUG_HOST_ROWS_VALID only the first frame_counts[b] rows of
+ * every utterance, the rest of the buffer untouched) and frame counts are copied
  * back, and the call returns after synchronising, so the host buffers are free
- * again.  Internally the batch is cut into up to 8 chunks of utterances that are
+ * again.  The longest rows of a chunk go by the copy engine while the kernel fetches
+ * the others, and valid feature rows are written by a kernel straight into a pinned
+ * (mapped) feature buffer, else by one copy per utterance.  Internally the batch is cut into up to 8 chunks of utterances that are
  * copied in, computed and copied out concurrently on three streams; speech rows
  * are copied only up to their length when that saves more than the extra copy
  * calls cost.  Host buffers should be pinned: copies then run asynchronously, and

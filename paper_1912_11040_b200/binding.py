@@ -41,7 +41,7 @@ class AugConfig(ctypes.Structure):
                 ("compression", ctypes.c_int32), ("max_batch", ctypes.c_int32),
                 ("max_samples", ctypes.c_int32), ("host_staging", ctypes.c_int32),
                 ("image_lattice", ctypes.c_int32), ("max_bank_samples", ctypes.c_int64),
-                ("vtlp_win", ctypes.c_int32), ("reserved_", ctypes.c_int32)]
+                ("vtlp_win", ctypes.c_int32), ("host_rows", ctypes.c_int32)]
 
 
 class AugDist(ctypes.Structure):
@@ -150,7 +150,7 @@ def make_config(cfg: dict, max_batch: int, max_samples: int, *, compression: int
                      max_batch=int(max_batch), max_samples=int(max_samples),
                      host_staging=int(bool(host_staging)), image_lattice=int(image_lattice),
                      max_bank_samples=int(max_bank_samples), vtlp_win=int(cfg.get("vtlp_win", 0)),
-                     reserved_=0)
+                     host_rows=int(cfg.get("host_rows", 0)))
 
 
 def aug_workspace_bytes(config: AugConfig) -> int:

@@ -3,6 +3,7 @@
 #include <new>
 #include <stdlib.h>
 #include <string.h>
+#include <algorithm>
 #include <vector>
 
 #include "common.cuh"
@@ -17,6 +18,12 @@ inline int64_t align_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
 // four samples, which the row stride always covers).  A small grid with many loads
 // in flight per thread does best (48 x 256 threads x 16 loads; larger grids were
 // slower), and the SMs stay free for the chunk that is being computed meanwhile.
+// Neither this kernel nor the copy engine fills the host link alone with rows of this
+// size (about 40 of 54 GB/s each), so a chunk's longest rows, AUG_DMA_SHARE_PCT percent
+// of its samples, go by the copy engine at the same time on a stream of their own.
+#ifndef AUG_DMA_SHARE_PCT
+#define AUG_DMA_SHARE_PCT 40
+#endif
 #ifndef AUG_COPY_CTAS
 #define AUG_COPY_CTAS 48
 #endif
@@ -24,10 +31,15 @@ inline int64_t align_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
 #define AUG_COPY_UNROLL 16
 #endif
 constexpr int COPY_CTAS = AUG_COPY_CTAS, COPY_THREADS = 256, COPY_UNROLL = AUG_COPY_UNROLL;
+#ifndef AUG_DMA_MIN_BYTES
+#define AUG_DMA_MIN_BYTES (512 << 10)
+#endif
+constexpr int64_t DMA_MIN_BYTES = AUG_DMA_MIN_BYTES;   // feature blocks of this size go back by the copy engine
 __global__ void __launch_bounds__(COPY_THREADS)
 copy_rows_kernel(const float4 *__restrict__ src, float4 *__restrict__ dst, int64_t stride4,
-                 const int *__restrict__ lengths, int b0, int b1) {
+                 const int *__restrict__ lengths, int b0, int b1, int below) {
     for (int b = b0; b < b1; ++b) {
+        if (lengths[b] >= below) continue;      // that row travels by the copy engine
         const int n4 = (max(lengths[b], 0) + 3) >> 2;
         const float4 *s = src + (int64_t)b * stride4;
         float4 *d = dst + (int64_t)b * stride4;
@@ -41,6 +53,20 @@ copy_rows_kernel(const float4 *__restrict__ src, float4 *__restrict__ dst, int64
             for (int u = 0; u < COPY_UNROLL; ++u)
                 if (i + u * step < n4) d[i + u * step] = v[u];
         }
+    }
+}
+
+// The first counts[b] feature rows (row4 groups of four floats each) of utterances
+// [b0, b1) from the device staging into the caller's mapped pinned buffer.
+__global__ void __launch_bounds__(COPY_THREADS)
+store_rows_kernel(const float4 *__restrict__ src, float4 *__restrict__ dst, int64_t utt4, int row4,
+                  const int *__restrict__ counts, int b0, int b1, int below) {
+    for (int b = b0; b < b1; ++b) {
+        if (counts[b] >= below) continue;       // that utterance travels by the copy engine
+        const int n4 = max(counts[b], 0) * row4;
+        const float4 *s = src + (int64_t)b * utt4;
+        float4 *d = dst + (int64_t)b * utt4;
+        for (int i = blockIdx.x * COPY_THREADS + threadIdx.x; i < n4; i += COPY_CTAS * COPY_THREADS) d[i] = s[i];
     }
 }
 
@@ -70,6 +96,7 @@ int check_config(const AugConfig *c) {
     if (!(c->sound_speed > 0.f) || !(c->log_floor > 0.f) || !isfinite(c->pad_value)) return AUG_EINVAL;
     if (c->compression != AUG_COMPRESS_LOG && c->compression != AUG_COMPRESS_POW_1_15) return AUG_EINVAL;
     if (c->image_lattice != AUG_LATTICE_TOTAL && c->image_lattice != AUG_LATTICE_CUBE) return AUG_EINVAL;
+    if (c->host_rows != AUG_HOST_ROWS_PADDED && c->host_rows != AUG_HOST_ROWS_VALID) return AUG_EINVAL;
     if (c->max_batch < 1 || c->max_batch > 65535 || c->max_samples < 1) return AUG_EINVAL;
     if (c->host_staging && c->max_bank_samples < 0) return AUG_EINVAL;
     if (c->vtlp_win < 0 || c->vtlp_win > 1024 || (c->vtlp_win & 3)) return AUG_EINVAL;
@@ -268,10 +295,13 @@ int aug_create(AugCtx **out, const AugConfig *cfg, void *cuda_stream) {
     }
     if (cfg->host_staging) {
         bool ok_s = cudaStreamCreateWithFlags(&ctx->s_h2d, cudaStreamNonBlocking) == cudaSuccess &&
+                    cudaStreamCreateWithFlags(&ctx->s_h2d2, cudaStreamNonBlocking) == cudaSuccess &&
+                    cudaEventCreateWithFlags(&ctx->ev_len, cudaEventDisableTiming) == cudaSuccess &&
                     cudaStreamCreateWithFlags(&ctx->s_d2h, cudaStreamNonBlocking) == cudaSuccess &&
                     cudaEventCreateWithFlags(&ctx->ev_start, cudaEventDisableTiming) == cudaSuccess;
         for (int i = 0; i < aug::HOST_CHUNKS && ok_s; ++i)
             ok_s = cudaEventCreateWithFlags(&ctx->ev_in[i], cudaEventDisableTiming) == cudaSuccess &&
+                   cudaEventCreateWithFlags(&ctx->ev_in2[i], cudaEventDisableTiming) == cudaSuccess &&
                    cudaEventCreateWithFlags(&ctx->ev_out[i], cudaEventDisableTiming) == cudaSuccess;
         if (!ok_s) {
             if (ctx->leff_seen) cudaFreeHost(ctx->leff_seen);
@@ -325,7 +355,13 @@ int aug_destroy(AugCtx *ctx) {
     if (ctx->s_h2d) {
         cudaStreamSynchronize(ctx->s_h2d);
         cudaStreamSynchronize(ctx->s_d2h);
+        if (ctx->s_h2d2) {
+            cudaStreamSynchronize(ctx->s_h2d2);
+            cudaStreamDestroy(ctx->s_h2d2);
+        }
+        if (ctx->ev_len) cudaEventDestroy(ctx->ev_len);
         for (int i = 0; i < aug::HOST_CHUNKS; ++i) {
+            if (ctx->ev_in2[i]) cudaEventDestroy(ctx->ev_in2[i]);
             cudaEventDestroy(ctx->ev_in[i]);
             cudaEventDestroy(ctx->ev_out[i]);
         }
@@ -510,7 +546,7 @@ int aug_pipeline_host(AugCtx *ctx, const float *speech_host, int64_t speech_stri
     // c is computed and chunk c-1 is copied out, on three streams tied by events.
     // Rows are copied only up to their length when the bytes saved outweigh the
     // cost of one copy call per row.
-    cudaStream_t sc = ctx->stream, si = ctx->s_h2d, so = ctx->s_d2h;
+    cudaStream_t sc = ctx->stream, si = ctx->s_h2d, si2 = ctx->s_h2d2, so = ctx->s_d2h;
     int64_t total = 0;
     for (int b = 0; b < B; ++b) total += lengths_host[b];
     const double saved_s = (double)((int64_t)B * speech_stride - total) * sizeof(float) / 40e9;
@@ -528,6 +564,11 @@ int aug_pipeline_host(AugCtx *ctx, const float *speech_host, int64_t speech_stri
                                 cudaMemcpyHostToDevice, si));
     AUG_CUDA_OK(cudaMemcpyAsync(ctx->st_lengths, lengths_host, sizeof(int) * (size_t)B,
                                 cudaMemcpyHostToDevice, si));
+    if (speech_alias) {
+        // the gather kernel's stream starts once the lengths are on the device
+        AUG_CUDA_OK(cudaEventRecord(ctx->ev_len, si));
+        AUG_CUDA_OK(cudaStreamWaitEvent(si2, ctx->ev_len, 0));
+    }
     if (bank_len > 0 && noise_bank_host) {
         AUG_CUDA_OK(cudaMemcpyAsync(ctx->st_bank, noise_bank_host, sizeof(float) * (size_t)bank_len,
                                     cudaMemcpyHostToDevice, si));
@@ -537,7 +578,21 @@ int aug_pipeline_host(AugCtx *ctx, const float *speech_host, int64_t speech_stri
     ctx->last_h2d = (int64_t)sizeof(AugUttParams) * B + (int64_t)sizeof(int) * B +
                     (int64_t)sizeof(float) * (noise_bank_host ? bank_len : 0) +
                     (int64_t)sizeof(float) * (ragged ? total : (int64_t)B * speech_stride);
-    ctx->last_d2h = (int64_t)sizeof(float) * B * T_max * M + (int64_t)sizeof(int) * B;
+    const bool valid_rows = ctx->cfg.host_rows == AUG_HOST_ROWS_VALID;
+    // frames per utterance as the device will count them (lengths are cut at the row stride)
+    auto frames_of = [&](int b) {
+        return std::min(aug_frame_count((int)std::min<int64_t>(lengths_host[b], speech_stride), ctx->cfg.win,
+                                        ctx->cfg.hop), T_max);
+    };
+    int64_t rows_out = (int64_t)B * T_max;
+    if (valid_rows) {
+        rows_out = 0;
+        for (int b = 0; b < B; ++b) rows_out += frames_of(b);
+    }
+    ctx->last_d2h = (int64_t)sizeof(float) * rows_out * M + (int64_t)sizeof(int) * B;
+    float *feats_alias = nullptr;
+    if (valid_rows && (M & 3) == 0 && aligned16(feats_host))
+        feats_alias = const_cast<float *>(mapped_alias(feats_host));
     int b0 = 0;
     int64_t done = 0;
     for (int c = 0; c < n_chunk; ++c) {
@@ -549,12 +604,33 @@ int aug_pipeline_host(AugCtx *ctx, const float *speech_host, int64_t speech_stri
         if (b1 == b0) continue;
         const int nb = b1 - b0;
         if (speech_alias) {
-            // (lengths reach the device on the same stream before this launch)
-            copy_rows_kernel<<<COPY_CTAS, COPY_THREADS, 0, si>>>(
+            // rows of at least `below` samples by the copy engine (the longest rows, up to its
+            // share of the chunk's samples), the others by the kernel, both at once
+            int below = 0x7fffffff;
+            if (AUG_DMA_SHARE_PCT > 0 && nb > 1) {
+                std::vector<int> len(lengths_host + b0, lengths_host + b1);
+                std::sort(len.begin(), len.end(), [](int a, int b) { return a > b; });
+                int64_t chunk_total = 0, acc = 0;
+                for (int v : len) chunk_total += v;
+                for (int v : len) {
+                    if ((acc + v) * 100 > chunk_total * AUG_DMA_SHARE_PCT) break;
+                    acc += v;
+                    below = v;
+                }
+            }
+            for (int b = b0; b < b1; ++b)
+                if (lengths_host[b] >= below)
+                    AUG_CUDA_OK(cudaMemcpyAsync(ctx->st_speech + (int64_t)b * speech_stride,
+                                                speech_host + (int64_t)b * speech_stride,
+                                                sizeof(float) * (size_t)lengths_host[b],
+                                                cudaMemcpyHostToDevice, si));
+            copy_rows_kernel<<<COPY_CTAS, COPY_THREADS, 0, si2>>>(
                 reinterpret_cast<const float4 *>(speech_alias), reinterpret_cast<float4 *>(ctx->st_speech),
-                speech_stride / 4, ctx->st_lengths, b0, b1);
+                speech_stride / 4, ctx->st_lengths, b0, b1, below);
             AUG_CUDA_OK(cudaGetLastError());
             ctx->launches++;
+            AUG_CUDA_OK(cudaEventRecord(ctx->ev_in2[c], si2));
+            AUG_CUDA_OK(cudaStreamWaitEvent(sc, ctx->ev_in2[c], 0));
         } else if (ragged) {
             for (int b = b0; b < b1; ++b)
                 if (lengths_host[b] > 0)
@@ -578,14 +654,51 @@ int aug_pipeline_host(AugCtx *ctx, const float *speech_host, int64_t speech_stri
         if (rc != AUG_OK) break;
         AUG_CUDA_OK(cudaEventRecord(ctx->ev_out[c], sc));
         AUG_CUDA_OK(cudaStreamWaitEvent(so, ctx->ev_out[c], 0));
-        AUG_CUDA_OK(cudaMemcpyAsync(feats_host + (int64_t)b0 * T_max * M, f_dev,
-                                    sizeof(float) * (size_t)nb * T_max * M, cudaMemcpyDeviceToHost, so));
+        if (feats_alias) {
+            // utterances with at least DMA_MIN_BYTES of features by the copy engine (it moves
+            // large blocks faster than stores from a kernel do), the others by the kernel
+            const int below = (int)std::min<int64_t>(0x7fffffff, (DMA_MIN_BYTES + 4 * M - 1) / (4 * M));
+            bool any_small = false;
+            for (int b = b0; b < b1; ++b) {
+                const int T = frames_of(b);
+                if (T >= below) {
+                    // utterances that fill all T_max rows run on into the next one: one copy
+                    int64_t rows = T;
+                    const int first = b;
+                    while (frames_of(b) == T_max && b + 1 < b1 && frames_of(b + 1) >= below)
+                        rows = (int64_t)(++b - first) * T_max + frames_of(b);
+                    AUG_CUDA_OK(cudaMemcpyAsync(feats_host + (int64_t)first * T_max * M,
+                                                ctx->st_feats + (int64_t)first * T_max * M,
+                                                sizeof(float) * (size_t)rows * M, cudaMemcpyDeviceToHost, so));
+                } else if (T > 0) {
+                    any_small = true;
+                }
+            }
+            if (any_small) {
+                store_rows_kernel<<<COPY_CTAS, COPY_THREADS, 0, so>>>(
+                    reinterpret_cast<const float4 *>(ctx->st_feats), reinterpret_cast<float4 *>(feats_alias),
+                    (int64_t)T_max * M / 4, M / 4, ctx->st_counts, b0, b1, below);
+                AUG_CUDA_OK(cudaGetLastError());
+                ctx->launches++;
+            }
+        } else if (valid_rows) {
+            for (int b = b0; b < b1; ++b)
+                if (frames_of(b) > 0)
+                    AUG_CUDA_OK(cudaMemcpyAsync(feats_host + (int64_t)b * T_max * M,
+                                                ctx->st_feats + (int64_t)b * T_max * M,
+                                                sizeof(float) * (size_t)frames_of(b) * M,
+                                                cudaMemcpyDeviceToHost, so));
+        } else {
+            AUG_CUDA_OK(cudaMemcpyAsync(feats_host + (int64_t)b0 * T_max * M, f_dev,
+                                        sizeof(float) * (size_t)nb * T_max * M, cudaMemcpyDeviceToHost, so));
+        }
         AUG_CUDA_OK(cudaMemcpyAsync(frame_counts_host + b0, ctx->st_counts + b0, sizeof(int) * (size_t)nb,
                                     cudaMemcpyDeviceToHost, so));
         b0 = b1;
     }
     // drain all three streams whatever happened above
-    const bool ok = cudaStreamSynchronize(si) == cudaSuccess && cudaStreamSynchronize(sc) == cudaSuccess &&
+    const bool ok = cudaStreamSynchronize(si) == cudaSuccess && cudaStreamSynchronize(si2) == cudaSuccess &&
+                    cudaStreamSynchronize(sc) == cudaSuccess &&
                     cudaStreamSynchronize(so) == cudaSuccess;
     if (rc != AUG_OK) return rc;
     return ok ? AUG_OK : AUG_ECUDA;

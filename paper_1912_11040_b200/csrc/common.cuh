@@ -90,7 +90,9 @@ struct AugCtx {
     int *st_counts;
     int64_t last_h2d, last_d2h;                // bytes the last aug_pipeline_host call copied
     cudaStream_t s_h2d, s_d2h;                 // copy streams of the host-buffer entry point
+    cudaStream_t s_h2d2;                       // the row-gather kernel's stream, beside the copy engine's
     cudaEvent_t ev_in[aug::HOST_CHUNKS], ev_out[aug::HOST_CHUNKS], ev_start;
+    cudaEvent_t ev_in2[aug::HOST_CHUNKS], ev_len;
     int64_t bank_resident;                     // samples of st_bank filled by aug_upload_noise_bank (0 = none)
 };
 

@@ -441,6 +441,46 @@ def test_host_entry_point_from_pinned_memory_matches_pageable():
     assert np.array_equal(counts.cpu().numpy(), cp) and np.max(np.abs(F.cpu().numpy() - Fp)) < 1e-3
 
 
+@pytest.mark.parametrize("config,batch,dur_scale", [(2, 12, 0.5), (5, 4, 0.4)])
+def test_host_entry_point_valid_rows_only(config, batch, dur_scale):
+    """With host_rows = VALID the host call writes the first frame_counts[b] rows of every
+    utterance and leaves the rest of the caller's buffer alone, from pinned memory (a kernel
+    writes short utterances, the copy engine those with 512 KB of features or more: the
+    second case) and from pageable memory (one copy per utterance); the bytes it reports
+    are those rows."""
+    import torch
+    w = small(config, batch=batch, dur_scale=dur_scale)
+    w.lengths[1] = 0
+    w.lengths[3] = w.lengths[3] // 2 + 1     # (second case: a full utterance followed by a long one, one copy)
+    if batch > 4:
+        w.lengths[4] = 1
+    dev_pad = Device(w, host_staging=True)
+    tab = np.ascontiguousarray(w.table)
+    Fp = np.full((w.B, dev_pad.T_max, dev_pad.M), np.nan, dtype=np.float32)
+    cp = np.full(w.B, -1, dtype=np.int32)
+    dev_pad.ctx.aug_pipeline_host(w.speech, w.stride, w.lengths, w.bank, w.bank.size, tab, w.B, Fp,
+                                  dev_pad.T_max, cp)
+    w.cfg["host_rows"] = 1
+    dev = Device(w, host_staging=True)
+    pin = lambda a: torch.from_numpy(a).pin_memory()
+    SENT = 123.25
+    Fh = torch.full((w.B, dev.T_max, dev.M), SENT).pin_memory()
+    ch = torch.full((w.B,), -1, dtype=torch.int32).pin_memory()
+    dev.ctx.aug_pipeline_host(pin(w.speech), w.stride, pin(w.lengths), pin(w.bank), w.bank.size,
+                              pin(tab.view(np.uint8).reshape(-1).copy()), w.B, Fh, dev.T_max, ch)
+    Fg = np.full((w.B, dev.T_max, dev.M), SENT, dtype=np.float32)
+    cg = np.full(w.B, -1, dtype=np.int32)
+    dev.ctx.aug_pipeline_host(w.speech, w.stride, w.lengths, w.bank, w.bank.size, tab, w.B, Fg, dev.T_max, cg)
+    for F, c in ((Fh.numpy(), ch.numpy()), (Fg, cg)):
+        assert np.array_equal(c, cp)
+        for b in range(w.B):
+            T = int(cp[b])
+            assert np.max(np.abs(F[b, :T] - Fp[b, :T]), initial=0.0) < 1e-3
+            assert np.all(F[b, T:] == SENT)
+    h2d, d2h = dev.ctx.aug_last_host_bytes()
+    assert d2h == 4 * int(cp.sum()) * dev.M + 4 * w.B
+
+
 def test_host_entry_point_with_an_uploaded_noise_bank():
     """A bank uploaded once serves later calls that pass no bank pointer; results and the
     bytes copied say so; a call with a bank of its own replaces the uploaded one."""

@@ -63,6 +63,11 @@ def test_strerror_and_workspace_size():
     assert binding.aug_workspace_bytes(cfg) > 0
     cfg.n_fft = 300
     assert binding.aug_workspace_bytes(cfg) == binding.AUG_EINVAL
+    cfg.n_fft = 512
+    cfg.host_rows = 1
+    assert binding.aug_workspace_bytes(cfg) > 0
+    cfg.host_rows = 2
+    assert binding.aug_workspace_bytes(cfg) == binding.AUG_EINVAL
 
 
 def test_validate_params():
