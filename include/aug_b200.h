@@ -356,7 +356,9 @@ int aug_upload_noise_bank(AugCtx *ctx, const float *noise_bank_host, int64_t ban
 /* -------------------------------------------------------------- measurement utilities
  * (instrumentation of this library; the paper has no counterpart) */
 
-#define AUG_N_STAGES 7 /* 0 impulse responses, 1 response lengths and spectra, 2 filterbank tables,
+#define AUG_N_STAGES 7 /* 0 impulse responses, 1 response lengths and spectra, 2 filterbank tables
+                            (on a stream of their own beside stages 0 and 1: their time is the
+                            time they took there and is not part of the sum of the others),
                           3 waveform warp (vtlp_win > 0) and block spectra of the audio (contexts
                             sized for responses of more than 8192 taps),
                           4 convolution, 5 waveform mix (only when requested), 6 features */

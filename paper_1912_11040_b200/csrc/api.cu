@@ -293,6 +293,17 @@ int aug_create(AugCtx **out, const AugConfig *cfg, void *cuda_stream) {
         }
         *ctx->leff_seen = 0;
     }
+    // The filterbank tables depend on the parameter table alone: aug_pipeline builds them on a
+    // stream of their own while the impulse responses are computed (without it, in line).
+    if (cudaStreamCreateWithFlags(&ctx->s_side, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming) != cudaSuccess) {
+        cudaGetLastError();
+        if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
+        if (ctx->s_side) cudaStreamDestroy(ctx->s_side);
+        ctx->s_side = nullptr;
+        ctx->ev_fork = ctx->ev_join = nullptr;
+    }
     if (cfg->host_staging) {
         bool ok_s = cudaStreamCreateWithFlags(&ctx->s_h2d, cudaStreamNonBlocking) == cudaSuccess &&
                     cudaStreamCreateWithFlags(&ctx->s_h2d2, cudaStreamNonBlocking) == cudaSuccess &&
@@ -352,6 +363,12 @@ int aug_destroy(AugCtx *ctx) {
         free(ctx->ev);
     }
 
+    if (ctx->s_side) {
+        cudaStreamSynchronize(ctx->s_side);
+        cudaEventDestroy(ctx->ev_fork);
+        cudaEventDestroy(ctx->ev_join);
+        cudaStreamDestroy(ctx->s_side);
+    }
     if (ctx->s_h2d) {
         cudaStreamSynchronize(ctx->s_h2d);
         cudaStreamSynchronize(ctx->s_d2h);
@@ -481,19 +498,38 @@ int aug_pipeline(AugCtx *ctx, const float *speech_dev, int64_t speech_stride,
         ev = ctx->ev + (size_t)ctx->ev_n * (2 * AUG_N_STAGES);
     auto t0 = [&](int stage, cudaStream_t st) { if (ev) cudaEventRecord(ev[2 * stage], st); };
     auto t1 = [&](int stage, cudaStream_t st) { if (ev) cudaEventRecord(ev[2 * stage + 1], st); };
-    // One stream: running the impulse-response chain beside the block spectra on a
-    // second stream was measured and gained nothing (both saturate the SMs' issue
-    // and shared-memory pipes), so the stages simply follow one another.
+    // Running the impulse-response chain beside the block spectra on a second stream was
+    // measured and gained nothing (both saturate the SMs' issue and shared-memory pipes), so
+    // those stages follow one another.  Only the small filterbank-table kernel, which needs
+    // nothing but the parameter table, runs beside them on the side stream.
     cudaStream_t sm = ctx->stream, ss = ctx->stream;
+    cudaStream_t st_mel = ctx->s_side ? ctx->s_side : ss;
+    if (ctx->s_side) {
+        AUG_CUDA_OK(cudaEventRecord(ctx->ev_fork, ss));     // after the caller's earlier work, this context's too
+        AUG_CUDA_OK(cudaStreamWaitEvent(ctx->s_side, ctx->ev_fork, 0));
+        t0(2, st_mel);
+        rc = launch_mel_tables(ctx, table_dev, B, st_mel);
+        t1(2, st_mel);
+        if (rc != AUG_OK) return rc;
+        AUG_CUDA_OK(cudaEventRecord(ctx->ev_join, ctx->s_side));
+    }
+    // every way out from here on first lets the context's stream wait for the side stream
+    auto joined = [&](int code) {
+        if (ctx->s_side && cudaStreamWaitEvent(sm, ctx->ev_join, 0) != cudaSuccess && code == AUG_OK)
+            return (int)AUG_ECUDA;
+        return code;
+    };
     t0(0, ss);
     rc = launch_rir(ctx, table_dev, B, ctx->rir, ss);
     t1(0, ss);
     t0(1, ss);
     if (rc == AUG_OK) rc = launch_rir_spectra(ctx, ctx->rir, table_dev, B, ss);
     t1(1, ss);
-    t0(2, ss);
-    if (rc == AUG_OK) rc = launch_mel_tables(ctx, table_dev, B, ss);
-    t1(2, ss);
+    if (!ctx->s_side) {
+        t0(2, ss);
+        if (rc == AUG_OK) rc = launch_mel_tables(ctx, table_dev, B, ss);
+        t1(2, ss);
+    }
 
     // waveform-domain warp first: the simulator then sees the warped speech (timed with stage 3)
     t0(3, sm);
@@ -507,17 +543,18 @@ int aug_pipeline(AugCtx *ctx, const float *speech_dev, int64_t speech_stride,
         rc = launch_convolve_prepare(ctx, speech_dev, speech_stride, lengths_dev, noise_bank_dev,
                                      bank_len, table_dev, B, max_len);
     t1(3, sm);
-    if (rc != AUG_OK) return rc;
+    if (rc != AUG_OK) return joined(rc);
     t0(4, sm);
     rc = launch_convolve_finish(ctx, speech_dev, speech_stride, lengths_dev, noise_bank_dev, bank_len,
                                 table_dev, B, max_len);
     t1(4, sm);
-    if (rc != AUG_OK) return rc;
+    if (rc != AUG_OK) return joined(rc);
     t0(5, sm);
     if (wave_out &&
         (rc = launch_mix(ctx, lengths_dev, table_dev, B, max_len, wave_out, speech_stride)) != AUG_OK)
-        return rc;
+        return joined(rc);
     t1(5, sm);
+    if ((rc = joined(AUG_OK)) != AUG_OK) return rc;
     t0(6, sm);
     rc = launch_fused_features(ctx, lengths_dev, table_dev, B, feats_dev, T_max, frame_counts_dev, max_len);
     t1(6, sm);

@@ -89,6 +89,8 @@ struct AugCtx {
     float *st_feats;       // [max_batch][t_cap][n_mel]
     int *st_counts;
     int64_t last_h2d, last_d2h;                // bytes the last aug_pipeline_host call copied
+    cudaStream_t s_side;                       // aug_pipeline builds the filterbank tables here, beside step 1
+    cudaEvent_t ev_fork, ev_join;
     cudaStream_t s_h2d, s_d2h;                 // copy streams of the host-buffer entry point
     cudaStream_t s_h2d2;                       // the row-gather kernel's stream, beside the copy engine's
     cudaEvent_t ev_in[aug::HOST_CHUNKS], ev_out[aug::HOST_CHUNKS], ev_start;

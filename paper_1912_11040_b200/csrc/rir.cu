@@ -72,10 +72,16 @@ __host__ __device__ constexpr size_t rir_smem_bytes(int threads, int L) {
            sizeof(float4) * threads + sizeof(float) * threads + sizeof(float) * (size_t)((L + 3) & ~3);
 }
 
-constexpr int THREADS = 512;      // 16 warps; two or three CTAs per multiprocessor
+#ifndef RIR_THREADS
+#define RIR_THREADS 512
+#endif
+#ifndef RIR_MINB
+#define RIR_MINB 3
+#endif
+constexpr int THREADS = RIR_THREADS;      // 16 warps; two or three CTAs per multiprocessor
 constexpr float HEADROOM_LOG2 = 6.f;   // full scale = 2^6 times the direct-path amplitude
 
-__global__ void __launch_bounds__(THREADS, 3)
+__global__ void __launch_bounds__(THREADS, RIR_MINB)
 rir_image_kernel(const AugUttParams *__restrict__ table, int S_max, int L, int half_w,
                  double fs_over_c, int max_order, int cube, float *__restrict__ rir, int *status) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
