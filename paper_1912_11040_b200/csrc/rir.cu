@@ -47,23 +47,10 @@ __device__ __forceinline__ float rcp_approx(float x) {
     return r;
 }
 
-// Add v, rounded to the nearest integer, to the int at shared address a + OFF if
-// |x| <= lim, as one predicated instruction (no branch around it).
+// Add iv to the int at shared address a + OFF (one instruction, no result wanted).
 template <int OFF>
-__device__ __forceinline__ void red_shared_within(unsigned a, float v, float x, float lim) {
-    asm volatile(
-        "{\n\t"
-        ".reg .pred p;\n\t"
-        ".reg .f32 ax;\n\t"
-        "abs.f32 ax, %2;\n\t"
-        "setp.le.f32 p, ax, %3;\n\t"
-        ".reg .s32 iv;\n\t"
-        "cvt.rni.s32.f32 iv, %1;\n\t"
-        "@p red.shared.add.s32 [%0+%4], iv;\n\t"
-        "}"
-        :
-        : "r"(a), "f"(v), "f"(x), "f"(lim), "n"(OFF)
-        : "memory");
+__device__ __forceinline__ void red_shared_add(unsigned a, int iv) {
+    asm volatile("red.shared.add.s32 [%0+%1], %2;" : : "r"(a), "n"(OFF), "r"(iv) : "memory");
 }
 
 // Bytes of dynamic shared memory of a CTA of `threads` threads for responses of L taps.
@@ -152,7 +139,9 @@ rir_image_kernel(const AugUttParams *__restrict__ table, int S_max, int L, int h
     }
     constexpr int NW = THREADS / 32;
     const unsigned h_addr = (unsigned)__cvta_generic_to_shared(h);
-    const unsigned inside = (unsigned)max(L - 2 * half_w, 0);   // first-tap samples whose whole window fits
+    // first-tap samples for which all 96 lane slots (81 of them taps) stay inside the response
+    const unsigned inside = (unsigned)max(L - 96, 0);
+    const bool mid_always = half_w >= 32;                       // taps 32..63 lie inside every window
     float4 *my4 = ring4 + warp * 32;
     float *my1 = ring1 + warp * 32;
 
@@ -231,10 +220,15 @@ rir_image_kernel(const AugUttParams *__restrict__ table, int S_max, int L, int h
                 // every tap of the window falls inside the response: no index checks, the
                 // three adds go to fixed offsets from one address
                 const unsigned a = h_addr + 4u * (unsigned)(n_first + lane);
+                // (a predicated reduction compiles to a branch around it: a tap outside the
+                // window adds zero instead; taps 32..63 are always inside it)
                 const float x0 = fj[0] - phi, x1 = fj[1] - phi, x2 = fj[2] - phi;
-                red_shared_within<0>(a, rcp_approx(x0) * fmaf(sj[0], P2, fmaf(cj[0], P1, P0)), x0, fhw);
-                red_shared_within<128>(a, rcp_approx(x1) * fmaf(sj[1], P2, fmaf(cj[1], P1, P0)), x1, fhw);
-                red_shared_within<256>(a, rcp_approx(x2) * fmaf(sj[2], P2, fmaf(cj[2], P1, P0)), x2, fhw);
+                const float v0 = rcp_approx(x0) * fmaf(sj[0], P2, fmaf(cj[0], P1, P0));
+                const float v1 = rcp_approx(x1) * fmaf(sj[1], P2, fmaf(cj[1], P1, P0));
+                const float v2 = rcp_approx(x2) * fmaf(sj[2], P2, fmaf(cj[2], P1, P0));
+                red_shared_add<0>(a, __float2int_rn(fabsf(x0) <= fhw ? v0 : 0.f));
+                red_shared_add<128>(a, __float2int_rn(mid_always ? v1 : (fabsf(x1) <= fhw ? v1 : 0.f)));
+                red_shared_add<256>(a, __float2int_rn(fabsf(x2) <= fhw ? v2 : 0.f));
             } else {
 #pragma unroll
                 for (int i = 0; i < 3; ++i) {
