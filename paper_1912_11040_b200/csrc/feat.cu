@@ -233,6 +233,8 @@ frames_kernel(const float *__restrict__ in_a, const float *__restrict__ in_b, in
     }
     float wv[E];
     window_values<E>(wv, win);
+    const int out_f0 = tid / M, out_m0 = tid - out_f0 * M;                   // first output element of this thread
+    const int step_f = FEAT_THREADS / M, step_m = FEAT_THREADS - step_f * M;  // and the stride to its next one
 
     for (int tile = 0; tile < TILES; ++tile) {
         const int t0 = run0 + tile * FT;
@@ -326,9 +328,16 @@ frames_kernel(const float *__restrict__ in_a, const float *__restrict__ in_b, in
                 }
             }
             __syncthreads();
+            // element i = frame * M + band sits at i + frame in the [FT][M+1] sums: walked without a division
+            int ff = out_f0, m = out_m0;
             for (int i = tid; i < nf * M; i += FEAT_THREADS) {
-                const int ff = i / M, m = i - ff * M;
-                orow[i] = compress(up_s[ff * (M + 1) + m] + dn_s[ff * (M + 1) + m + 1], floor_v, comp);
+                orow[i] = compress(up_s[i + ff] + dn_s[i + ff + 1], floor_v, comp);
+                ff += step_f;
+                m += step_m;
+                if (m >= M) {
+                    m -= M;
+                    ++ff;
+                }
             }
         }
         __syncthreads();   // ptile, the interval sums (= the transform buffers) and chunk are reused by the next tile
