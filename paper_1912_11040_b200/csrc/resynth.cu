@@ -28,7 +28,10 @@ constexpr int E = 16;                 // points per thread
 constexpr int GROUP = K / E;          // 64 threads per transform
 constexpr int NGROUP = 4;
 constexpr int RS_THREADS = GROUP * NGROUP;
-constexpr int HB = 16;                // hops of output per CTA
+#ifndef RS_HB
+#define RS_HB 13
+#endif
+constexpr int HB = RS_HB;             // hops of output per CTA: 13 + 3 frames = 8 pairs, two full rounds of the four groups
 constexpr int NF = HB + 3;            // frames that cover them
 constexpr int XB = padded_points(K);
 
@@ -72,7 +75,7 @@ vtlp_positions_kernel(const AugUttParams *__restrict__ table, int *__restrict__ 
     }
 }
 
-__global__ void __launch_bounds__(RS_THREADS)
+__global__ void __launch_bounds__(RS_THREADS, 2)
 vtlp_resynth_kernel(const float *__restrict__ speech, int64_t stride, const int *__restrict__ lengths,
                     const int *__restrict__ k0_tab, const float *__restrict__ fr_tab, int win,
                     const float2 *__restrict__ tw, float *__restrict__ out, int64_t out_stride, int n_cap) {
@@ -114,7 +117,7 @@ vtlp_resynth_kernel(const float *__restrict__ speech, int64_t stride, const int 
     float acc[OWN];
 #pragma unroll
     for (int u = 0; u < OWN; ++u) acc[u] = 0.f;
-    const float inv_k = 1.f / (float)K;
+    const float inv_k = 1.f / (float)K, inv_hop = 1.f / (float)hop;
 
     for (int round = 0; round * NGROUP < NPAIR; ++round) {
         const int pr = round * NGROUP + grp;
@@ -152,24 +155,24 @@ vtlp_resynth_kernel(const float *__restrict__ speech, int64_t stride, const int 
             fft1024_in_place(W, tg, tw, gsync);               // W[n] = (imaginary, real) of the inverse, times K
         }
         __syncthreads();
-        // what this round's frames add to the owned samples: sample i of the CTA sits at
-        // n = i + (3 - slot) hop of the frame in `slot`
+        // What this round's frames add to the owned samples.  Sample i of the CTA lies in hop
+        // q = i / hop at offset r and is covered by the four frames in slots q .. q + 3, at
+        // n = r + (3 - d) hop of slot q + d; this round holds slots 8 round .. 8 round + 7
+        // (group g: slots 2 g and 2 g + 1, in the imaginary and real part of its buffer).
 #pragma unroll
         for (int u = 0; u < OWN; ++u) {
             const int i = tid + u * RS_THREADS;
             if (i < HB * hop) {
+                const int q = (int)(((float)i + 0.5f) * inv_hop);      // exact: i + 1/2 is never a multiple of hop
+                const int r = i - q * hop;
                 float sum = 0.f;
-                for (int g = 0; g < NGROUP; ++g) {
-                    const int slot = 2 * (round * NGROUP + g);
-                    const float2 *Wg = wbuf + g * XB;
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        const int sl = slot + h, t = t0 - 3 + sl;
-                        const int n = i + (3 - sl) * hop;
-                        if (sl < NF && t >= 0 && t < T && n >= 0 && n < win) {
-                            const float2 z = Wg[pad0(n)];
-                            sum = fmaf(wn[n], h ? z.x : z.y, sum);
-                        }
+                for (int d = 0; d < 4; ++d) {
+                    const int gl = q + d - 2 * NGROUP * round, t = t0 - 3 + q + d;
+                    if ((unsigned)gl < (unsigned)(2 * NGROUP) && t >= 0 && t < T) {
+                        const int n = r + (3 - d) * hop;
+                        const float *Wf = reinterpret_cast<const float *>(wbuf + (gl >> 1) * XB);
+                        sum = fmaf(wn[n], Wf[2 * n + 1 - (gl & 1)], sum);
                     }
                 }
                 acc[u] = fmaf(sum, inv_k, acc[u]);
