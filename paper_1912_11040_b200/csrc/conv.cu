@@ -460,6 +460,26 @@ constexpr int NQ2 = N2 / 2 / CT;       // slot pairs per thread and buffer
 __device__ __forceinline__ void load_segment4(float2 (*va)[E], float2 (*vb)[E],
                                               const float *__restrict__ x, bool looped, int nlen,
                                               int base, int N, int t, const float *xend) {
+    // A segment that lies inside the utterance (most do), and for a looped stretch inside one
+    // period of it on 16-byte boundaries, needs no test per group: the same for the whole CTA.
+    if (base >= 0 && base + F2 <= N) {
+        int m0 = base;
+        bool plain = !looped;
+        if (looped && (nlen & 3) == 0 && (reinterpret_cast<uintptr_t>(x) & 15) == 0) {
+            m0 = base % nlen;
+            plain = m0 + F2 <= nlen;
+        }
+        if (plain) {
+            const float4 *x4 = reinterpret_cast<const float4 *>(x + m0) + t;
+#pragma unroll
+            for (int r = 0; r < E; ++r) {
+                const float4 z = __ldg(x4 + CT * r);
+                va[0][r] = make_float2(z.x, z.y);
+                vb[0][r] = make_float2(z.z, z.w);
+            }
+            return;
+        }
+    }
     if (!looped) {
 #pragma unroll
         for (int r = 0; r < E; ++r) {
