@@ -919,6 +919,21 @@ convolve_fused2_kernel(const float *__restrict__ speech, int64_t stride,
         const bool want_energy = is_speech || s == last_noise;
         float *dst = (is_speech ? ys : vv) + (int64_t)utt * ws_stride + (int64_t)b * ob;
         float e2sum = 0.f;
+        if (n_left >= ob) {
+            // a whole block of outputs (the same for the CTA): no test per group
+#pragma unroll 4
+            for (int j = t; m0 + j < N2; j += CT) {
+                const float2 za = A[pad0(m0 + j)], zb = Bf[pad0(m0 + j)];
+                float4 y = make_float4(za.y, za.x, zb.y, zb.x);
+                float4 *p = reinterpret_cast<float4 *>(dst + 4 * j);
+                if (add) {
+                    const float4 o = *p;
+                    y = make_float4(y.x + o.x, y.y + o.y, y.z + o.z, y.w + o.w);
+                }
+                *p = y;
+                e2sum += y.x * y.x + y.y * y.y + y.z * y.z + y.w * y.w;
+            }
+        } else
 #pragma unroll 4
         for (int j = t; m0 + j < N2; j += CT) {
             const float2 za = A[pad0(m0 + j)], zb = Bf[pad0(m0 + j)];
