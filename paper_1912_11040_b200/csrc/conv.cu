@@ -122,6 +122,22 @@ __device__ __forceinline__ void mac_pair(float2 &acc_a, float2 &acc_b, float2 a,
 // its stretch of the bank end to end (x[i mod nlen]).  Outside [0, N): zero.
 __device__ __forceinline__ void load_segment(float2 (*v)[E], const float *__restrict__ x, bool looped,
                                              int nlen, int base, int N, int t) {
+    // A segment inside the utterance, and for a looped stretch inside one period of it on
+    // 8-byte boundaries, needs no test per pair (the same for the whole CTA).
+    if (base >= 0 && base + 2 * BLK <= N) {
+        int m0 = base;
+        bool plain = !looped;
+        if (looped && (nlen & 1) == 0 && (reinterpret_cast<uintptr_t>(x) & 7) == 0) {
+            m0 = base % nlen;
+            plain = (m0 & 1) == 0 && m0 + 2 * BLK <= nlen;
+        }
+        if (plain) {
+            const float2 *x2 = reinterpret_cast<const float2 *>(x + m0) + t;
+#pragma unroll
+            for (int r = 0; r < E; ++r) v[0][r] = __ldg(x2 + CT * r);
+            return;
+        }
+    }
     if (!looped) {
 #pragma unroll
         for (int r = 0; r < E; ++r) {
